@@ -1,0 +1,274 @@
+"""TEST INFRASTRUCTURE -- plain fp64 CPU statement of the Flag Aggregator step.
+
+Nothing in the product path may import this file: it exists so that tests, the
+smoke check and the benchmark's CPU-baseline leg have something slow and
+readable to compare the CUDA path against.  It shares no code with the CUDA
+path and works directly on n-dimensional vectors.
+
+What it computes (Flag Aggregator paper, arXiv 2302.05865):
+
+  * gradients g_1..g_p in R^n, the rows of the worker-major array G (the
+    paper's gradient matrix, Section 2.1, is its transpose);
+  * the subspace Y (n x m, orthonormal columns) that the iteratively
+    reweighted least-squares ("flag mean") procedure of Algorithm 1 reaches
+    for the objective of Eq. (5) with the data-dependent regulariser (2) of
+    Section 2.3,
+        A(Y) = sum_i sqrt(1 - ||Y^T g_i||^2 / ||g_i||^2)
+             + lam/(p-1) * sum_{i != j} sqrt(1 - ||Y^T (g_i-g_j)||^2 / D_ij^2),
+    D_ij^2 = ||g_i - g_j||^2;
+  * the update direction d = (1/p) Y Y^T G 1 of Algorithm 1.
+
+How each round is taken (the paper names the procedure but prints no update
+formula; this is the reading used, each item listed in the design notes):
+
+  * round 1 uses uniform weights, so it is PCA of the gradient matrix
+    (appendix "Experiments with other Byzantine attacks or baselines");
+  * later rounds reweight every square-root term of the objective by
+    1 / (normaliser * sqrt(term's current value)) -- for the data terms this
+    is -d_i of the appendix equation defining g-tilde_i -- and take the m
+    leading eigenvectors of
+        C = sum_i w_i g_i g_i^T + sum_{i != j} w_ij (g_i-g_j)(g_i-g_j)^T,
+    i.e. one weighted PCA;
+  * the value under each square root is evaluated as the relative squared
+    residual ||x - Y Y^T x||^2 / ||x||^2, which equals 1 - ||Y^T x||^2/||x||^2
+    for orthonormal Y (Section 2.1) and does not cancel;
+  * sqrt(.) in a weight is floored at EPS; zero gradients and identical pairs
+    carry weight 0 and contribute 0 to the objective; eigen-directions whose
+    eigenvalue is <= RANK_REL * largest are left out of Y;
+  * exactly `iters` rounds are run (no early exit).
+
+Two ways of getting the eigenvectors of C are provided and tested against
+each other: "literal" builds the n x n matrix C term by term (small n only);
+"svd" uses C = B B^T with B = G^T M^(1/2), M = diag(w) + sum w_ij (e_i-e_j)
+(e_i-e_j)^T, and takes the left singular vectors of the n x p matrix B.
+
+Parity pins (tests/test_oracle_pins.py): mean recovery, orthonormality and
+ratio range, PCA special case, worker-permutation and scaling invariance,
+monotone descent, first-order stationarity of Eq. (5) at the fixed point by
+finite differences, the right-multiplication form of the appendix KKT section,
+brute force over the Grassmannian for n <= 4, the Kronecker/trace identity of
+Lemma "Equivalence of Objective Functions", m = p, literal vs svd.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+EPS = 1e-6              # floor on sqrt(1 - v) inside a weight
+ZERO_NORM_REL = 1e-30   # ||g_i||^2 <= this * max_k ||g_k||^2  => zero gradient
+SAME_PAIR_REL = 1e-12   # D_ij^2 <= this * (||g_i||^2 + ||g_j||^2) => identical pair
+RANK_REL = 1e-12        # eigenvalue <= this * largest => direction dropped from Y
+
+
+# -- plain definitions -------------------------------------------------------
+
+def inner_products(G: np.ndarray) -> np.ndarray:
+    """K_ij = <g_i, g_j> (Section 2.1: ||g_i||^2 on the diagonal)."""
+    G = np.asarray(G, dtype=np.float64)
+    return G @ G.T
+
+
+def pair_sqdist(G: np.ndarray) -> np.ndarray:
+    """D_ij^2 = ||g_i - g_j||^2 from the difference vector (Section 2.3, item 2)."""
+    G = np.asarray(G, dtype=np.float64)
+    p = G.shape[0]
+    D2 = np.zeros((p, p))
+    for i in range(p):
+        for j in range(i + 1, p):
+            diff = G[i] - G[j]
+            D2[i, j] = D2[j, i] = float(diff @ diff)
+    return D2
+
+
+def residual_ratio(Y: np.ndarray, x: np.ndarray) -> float:
+    """1 - ||Y^T x||^2/||x||^2 written as ||x - Y Y^T x||^2 / ||x||^2."""
+    res = x - Y @ (Y.T @ x)
+    return float(res @ res) / float(x @ x)
+
+
+def _classify(G):
+    p = G.shape[0]
+    norms = np.einsum("ij,ij->i", G, G)
+    top = float(norms.max()) if p else 0.0
+    zero = norms <= ZERO_NORM_REL * top
+    return norms, zero
+
+
+def _pairs(G, norms, lam):
+    """D_ij^2 and the mask of pairs that take part (i != j, not identical)."""
+    p = G.shape[0]
+    if lam <= 0 or p < 2:
+        return np.zeros((p, p)), np.zeros((p, p), dtype=bool)
+    D2 = pair_sqdist(G)
+    active = D2 > SAME_PAIR_REL * (norms[:, None] + norms[None, :])
+    np.fill_diagonal(active, False)
+    return D2, active
+
+
+def residuals(G, Y):
+    """Rows r_i = g_i - Y Y^T g_i (what the subspace does not reconstruct, Section 2.1)."""
+    return G - (G @ Y) @ Y.T
+
+
+def term_values(G, Y, lam, norms=None, zero=None, D2=None, active=None):
+    """u_i and u_ij: the quantities under the square roots of Eq. (5).
+
+    The projector is linear, so the residual of g_i - g_j is r_i - r_j.
+    """
+    G = np.asarray(G, dtype=np.float64)
+    p = G.shape[0]
+    if norms is None:
+        norms, zero = _classify(G)
+    if D2 is None:
+        D2, active = _pairs(G, norms, lam)
+    R = residuals(G, Y)
+    u = np.zeros(p)
+    for i in range(p):
+        if not zero[i]:
+            u[i] = float(R[i] @ R[i]) / norms[i]
+    U = np.zeros((p, p))
+    if lam > 0:
+        for i in range(p):
+            for j in range(i + 1, p):
+                if active[i, j]:
+                    diff = R[i] - R[j]
+                    U[i, j] = U[j, i] = float(diff @ diff) / D2[i, j]
+    return u, U
+
+
+def objective(G, Y, lam) -> float:
+    """A(Y) of Eq. (5) with regulariser (2); the pair sum runs over ordered pairs."""
+    G = np.asarray(G, dtype=np.float64)
+    p = G.shape[0]
+    u, U = term_values(G, Y, lam)
+    val = float(np.sum(np.sqrt(np.maximum(u, 0.0))))
+    if lam > 0 and p > 1:
+        val += lam / (p - 1) * float(np.sum(np.sqrt(np.maximum(U, 0.0))))
+    return val
+
+
+# -- one weighted PCA ----------------------------------------------------------
+
+def _keep(evals_desc, m):
+    if evals_desc.size == 0 or evals_desc[0] <= 0:
+        return 0
+    return int(np.sum(evals_desc[:m] > RANK_REL * evals_desc[0]))
+
+
+def weighted_pca_literal(G, w, W, m):
+    """Leading eigenvectors of C built term by term as an n x n matrix."""
+    p, n = G.shape
+    C = np.zeros((n, n))
+    for i in range(p):
+        if w[i] != 0.0:
+            C += w[i] * np.outer(G[i], G[i])
+    for i in range(p):
+        for j in range(p):
+            if i != j and W[i, j] != 0.0:
+                x = G[i] - G[j]
+                C += W[i, j] * np.outer(x, x)
+    evals, evecs = np.linalg.eigh(C)
+    evals, evecs = evals[::-1], evecs[:, ::-1]
+    k = _keep(evals, min(m, n))
+    return evecs[:, :k], evals
+
+
+def pair_weight_matrix(w, W):
+    """M with C = G^T M G for worker-major G: diag(w) + sum_{i != j} W_ij (e_i-e_j)(e_i-e_j)^T."""
+    p = w.shape[0]
+    M = np.diag(np.asarray(w, dtype=np.float64))
+    for i in range(p):
+        for j in range(p):
+            if i != j and W[i, j] != 0.0:
+                M[i, i] += W[i, j]
+                M[j, j] += W[i, j]
+                M[i, j] -= W[i, j]
+                M[j, i] -= W[i, j]
+    return M
+
+
+def weighted_pca_svd(G, w, W, m):
+    """Same subspace from the thin SVD of B = G^T M^(1/2) (n x p)."""
+    p, n = G.shape
+    if np.any(W != 0.0):
+        M = pair_weight_matrix(w, W)
+        e, E = np.linalg.eigh(M)
+        S = E * np.sqrt(np.maximum(e, 0.0))[None, :]      # S S^T = M
+        B = G.T @ S
+    else:
+        B = G.T * np.sqrt(w)[None, :]
+    Uleft, s, _ = np.linalg.svd(B, full_matrices=False)
+    evals = s * s
+    k = _keep(evals, min(m, n))
+    return Uleft[:, :k], evals
+
+
+# -- the iteration -------------------------------------------------------------
+
+def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False):
+    """Run `iters` IRLS rounds and return the aggregate.
+
+    G      : (p, n) array, rows are worker gradients (converted to float64)
+    returns: dict with d (n,), Y (n, k<=m), u (p,), w (p,) last data weights,
+             objective (list, one per round), evals (last round, descending),
+             and with history=True the list of Y per round.
+    """
+    G = np.asarray(G, dtype=np.float64)
+    p, n = G.shape
+    if not (1 <= m <= p):
+        raise ValueError("need 1 <= m <= p")
+    if iters < 1 or lam < 0:
+        raise ValueError("need iters >= 1 and lam >= 0")
+    norms, zero = _classify(G)
+    D2, active = _pairs(G, norms, lam)
+    coef = lam / (p - 1) if (lam > 0 and p > 1) else 0.0
+    pca = weighted_pca_literal if method == "literal" else weighted_pca_svd
+
+    if np.all(zero):                       # every gradient is zero: nothing to span
+        return dict(d=np.zeros(n), Y=np.zeros((n, 0)), u=np.zeros(p), w=np.zeros(p),
+                    objective=[0.0] * iters, evals=np.zeros(p), Ys=[])
+
+    u = np.zeros(p)
+    U = np.zeros((p, p))
+    objs, Ys = [], []
+    for t in range(1, iters + 1):
+        w = np.zeros(p)
+        W = np.zeros((p, p))
+        if t == 1:
+            w[~zero] = 1.0
+            W[active] = coef
+        else:
+            r = np.sqrt(np.maximum(u, 0.0))
+            w[~zero] = 1.0 / (norms[~zero] * np.maximum(r[~zero], eps))
+            if coef > 0:
+                R = np.sqrt(np.maximum(U, 0.0))
+                W[active] = coef / (D2[active] * np.maximum(R[active], eps))
+        Y, evals = pca(G, w, W, m)
+        u, U = term_values(G, Y, lam, norms, zero, D2, active)
+        obj = float(np.sum(np.sqrt(np.maximum(u, 0.0))))
+        if coef > 0:
+            obj += coef * float(np.sum(np.sqrt(np.maximum(U, 0.0))))
+        objs.append(obj)
+        if history:
+            Ys.append(Y)
+    d = Y @ (Y.T @ G.sum(axis=0)) / p
+    return dict(d=d, Y=Y, u=u, w=w, objective=objs, evals=evals, Ys=Ys)
+
+
+# -- comparison helpers ----------------------------------------------------------
+
+def principal_angles(Ya, Yb) -> np.ndarray:
+    """asin of the singular values of (I - Ya Ya^T) Yb, largest first (radians)."""
+    Ya = np.asarray(Ya, dtype=np.float64)
+    Yb = np.asarray(Yb, dtype=np.float64)
+    if Ya.shape[1] == 0 or Yb.shape[1] == 0:
+        return np.zeros(0)
+    R = Yb - Ya @ (Ya.T @ Yb)
+    s = np.linalg.svd(R, compute_uv=False)
+    return np.arcsin(np.clip(s, 0.0, 1.0))
+
+
+def rel_l2(a, b) -> float:
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    den = float(np.linalg.norm(b))
+    return float(np.linalg.norm(a - b)) / den if den > 0 else float(np.linalg.norm(a))
