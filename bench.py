@@ -1,0 +1,312 @@
+#!/usr/bin/env python
+"""Benchmark of the Flag Aggregator step (Gram pass -> IRLS -> output pass) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+One step = one whole aggregation of a seeded synthetic gradient set (default: the p=15,
+n=11,173,962 fp32 workload the headline metric is quoted on).  Prints ONE JSON line.
+With N > 1 (under torchrun) every rank aggregates its own independent replica of the workload
+(the step has no cross-GPU exchange), so the value is N times the per-GPU rate: weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synthetic_inputs as si  # noqa: E402
+
+METRIC = "aggregations/sec at p=15, n=11.2M (whole Flag Aggregator step)"
+UNIT = "aggregations/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (file absent)"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs (read-only)."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.file.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        nums = [d.get("num_threads", 1) for d in threadpool_info() if d.get("user_api") == "blas"]
+        if nums:
+            return max(nums)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def time_oracle(w: si.Workload, n_sample: int, repeats: int = 1):
+    """Oracle, as it stands, on the same recipe at n_sample columns; returns seconds per sample run."""
+    from oracle import fa_oracle as fo
+    ws = w.scaled(n_sample)
+    G = si.to_float64(si.generate(ws))
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        fo.fa_aggregate(G, w.m, w.lam, w.iters)
+        times.append(time.perf_counter() - t0)
+    return min(times)
+
+
+def run_reference(args, w):
+    """The CPU oracle as the reference arm: each step is the oracle on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import fa_oracle as fo
+    n_sample = max(4096, w.n // 64)
+    ws = w.scaled(n_sample)
+    G = si.to_float64(si.generate(ws))
+    for _ in range(args.warmup):
+        fo.fa_aggregate(G, w.m, w.lam, w.iters)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        fo.fa_aggregate(G, w.m, w.lam, w.iters)
+    dt = (time.perf_counter() - t0) / args.steps
+    scale = w.n / n_sample
+    value = 1.0 / (dt * scale)
+    sample = f"{w.name} recipe at n={n_sample} (1/{scale:.1f} of the columns), cost scaled linearly in n"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * scale * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "p": w.p, "n": w.n, "m": w.m, "lambda": w.lam, "iters": w.iters},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(si.WORKLOADS))
+    ap.add_argument("--n", type=int, default=None, help="override the gradient length (profiling small cases)")
+    ap.add_argument("--buffers", type=int, default=3, help="independent copies of G rotated between steps")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    w = si.WORKLOADS[args.workload]
+    if args.n:
+        w = w.scaled(args.n)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2302_05865_b200 as fa
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the aggregation has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- inputs: generated once on the host, R copies on the device (addresses differ, so a
+    # step never finds its gradients in L2 from the previous step); every copy is > L2 at cfg2
+    G_np = si.generate(w)
+    host = torch.from_numpy(G_np.view(np.int16)).view(torch.bfloat16) if w.dtype == "bf16" else torch.from_numpy(G_np)
+    nbuf = max(1, args.buffers)
+    Gs = [host.cuda() for _ in range(nbuf)]
+    out = torch.empty(w.n, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wsb = fa.new_workspace(Gs[0], w.m)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        fa.fa_aggregate(Gs[i % nbuf], w.m, w.lam, w.iters, out=out, ws=wsb, status=status, stream=stream)
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {int(status.item())} after the timed region")
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * 1e3 / ms_per_step
+
+    # ---- per-kernel times, same buffers and stream, CUDA events around single launches
+    def time_call(fn, reps):
+        e0 = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]
+        e1 = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]
+        for i in range(reps):
+            e0[i].record(stream)
+            fn(i)
+            e1[i].record(stream)
+        torch.cuda.synchronize()
+        return statistics.mean(a.elapsed_time(b) for a, b in zip(e0, e1))
+
+    reps = max(10, min(args.steps, 50))
+    K = torch.empty((w.p, w.p), dtype=torch.float64, device="cuda")
+    cvec = torch.full((w.p,), 1.0 / w.p, dtype=torch.float32, device="cuda")
+    fa.fa_gram(Gs[0], K=K, ws=wsb); fa.fa_combine(Gs[0], cvec, out=out); fa.fa_irls(K, w.m, w.lam, w.iters, c_out=cvec)
+    torch.cuda.synchronize()
+    t_gram = time_call(lambda i: fa.fa_gram(Gs[i % nbuf], K=K, ws=wsb, stream=stream), reps)
+    t_comb = time_call(lambda i: fa.fa_combine(Gs[i % nbuf], cvec, out=out, stream=stream), reps)
+    t_irls = time_call(lambda i: fa.fa_irls(K, w.m, w.lam, w.iters, c_out=cvec, stream=stream), reps)
+
+    peak, peak_src = measured_peaks()
+    gram_bytes = w.p * w.n * w.itemsize
+    comb_bytes = w.p * w.n * w.itemsize + 4 * w.n
+    gram_gbs = gram_bytes / (t_gram * 1e-3) / 1e9
+    comb_gbs = comb_bytes / (t_comb * 1e-3) / 1e9
+    step_gbs = w.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point (pinned host memory both ways)
+    e2e = None
+    if not args.no_e2e:
+        Gh = host.pin_memory()
+        outh = torch.empty(w.n, dtype=torch.float32).pin_memory()
+        sth = torch.zeros(1, dtype=torch.int32).pin_memory()
+        k_e2e = max(3, min(args.steps, 10))
+        for _ in range(2):
+            fa.fa_aggregate_host(Gh, w.m, w.lam, w.iters, outh, Gs[0], out, wsb, sth, status, stream=stream)
+        barrier()
+        ev0.record(stream)
+        for i in range(k_e2e):
+            fa.fa_aggregate_host(Gh, w.m, w.lam, w.iters, outh, Gs[i % nbuf], out, wsb, sth, status, stream=stream)
+        ev1.record(stream)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * 1e3 / (ms / k_e2e), "unit": UNIT,
+               "h2d_bytes_per_step": int(gram_bytes), "d2h_bytes_per_step": int(4 * w.n + 4),
+               "steps": k_e2e, "ms_per_step": ms / k_e2e}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_sample = max(4096, w.n // 8)
+        t_s = time_oracle(w, n_sample)
+        scale = w.n / n_sample
+        cpu = {"value": 1.0 / (t_s * scale), "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+               "sample": f"{w.name} recipe at n={n_sample} (1/{scale:.1f} of the columns), {t_s:.1f} s measured, "
+                         f"cost scaled linearly in n"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "p": w.p, "f": w.f, "n": w.n, "m": w.m, "lambda": w.lam, "iters": w.iters,
+                   "storage": w.dtype, "l2": f"inputs larger than L2; {nbuf} device copies of G rotated between steps",
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+        "roofline": {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
+                     "unit": "GB/s", "frac": gram_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "bytes_per_launch": int(gram_bytes), "ms_per_launch": t_gram},
+        "kernels": {"gram_ms": t_gram, "irls_ms": t_irls, "combine_ms": t_comb,
+                    "combine_gbs": comb_gbs, "combine_frac": comb_gbs / peak},
+        "step_hbm": {"algorithmic_bytes": int(w.algorithmic_bytes), "achieved_gbs": step_gbs,
+                     "frac_of_measured": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / 8000.0},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": 3 * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,168 @@
+// C ABI of the library (declared in include/fa.h): argument checks, workspace carving, launches.
+// Nothing here allocates, frees or synchronises.
+#include <math.h>
+#include <stdint.h>
+
+#include "../../include/fa.h"
+#include "fa_kernels.h"
+
+namespace fa {
+
+int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  if (cached[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    cached[dev] = v;
+  }
+  return cached[dev];
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t round_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Workspace {
+  double* partials;
+  double* Kbuf;
+  float* c;
+  size_t total;
+};
+
+Workspace carve_ws(void* ws, int p, long long n, int dtype) {
+  Workspace w{};
+  size_t off = 0;
+  char* base = static_cast<char*>(ws);
+  w.partials = reinterpret_cast<double*>(base + off);
+  off += round_up(gram_partials_bytes(p, n, dtype));
+  w.Kbuf = reinterpret_cast<double*>(base + off);
+  off += round_up((size_t)p * p * sizeof(double));
+  w.c = reinterpret_cast<float*>(base + off);
+  off += round_up(FA_MAX_P * sizeof(float));
+  w.total = off;
+  return w;
+}
+
+bool shape_ok(int p, long long n, int dtype) {
+  return p >= 1 && p <= FA_MAX_P && n >= 1 && (dtype == FA_F32 || dtype == FA_BF16);
+}
+
+bool aligned(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+
+}  // namespace
+}  // namespace fa
+
+extern "C" {
+
+const char* fa_error_string(int code) {
+  switch (code) {
+    case FA_OK: return "ok";
+    case FA_ERR_ARG: return "invalid argument";
+    case FA_ERR_ALIGN: return "misaligned pointer";
+    case FA_ERR_WORKSPACE: return "workspace too small";
+    case FA_ERR_CUDA: return "CUDA launch failed";
+    default: return "unknown error code";
+  }
+}
+
+int fa_workspace_bytes(int p, long long n, int m, int dtype, size_t* bytes) {
+  (void)m;
+  if (!bytes || !fa::shape_ok(p, n, dtype)) return FA_ERR_ARG;
+  *bytes = fa::carve_ws(nullptr, p, n, dtype).total;
+  return FA_OK;
+}
+
+int fa_gram(const void* G, int dtype, int p, long long n, double* K, void* ws, size_t ws_bytes, void* stream) {
+  if (!G || !K || !ws || !fa::shape_ok(p, n, dtype)) return FA_ERR_ARG;
+  if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(K, 8) || !fa::aligned(ws, 16)) return FA_ERR_ALIGN;
+  fa::Workspace w = fa::carve_ws(ws, p, n, dtype);
+  if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int nblocks = 0;
+  if (fa::launch_gram_partials(G, dtype, p, n, w.partials, nullptr, st, &nblocks) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_reduce_partials(w.partials, nblocks, p, K, st) != cudaSuccess) return FA_ERR_CUDA;
+  return FA_OK;
+}
+
+int fa_irls_step(const double* K, int p, int m, double lambda, int first, double* A, double* w, double* objective,
+                 int* status, void* stream) {
+  if (!K || !A || !w || p < 1 || p > FA_MAX_P || m < 1 || m > p || !(lambda >= 0.0) || isinf(lambda)) return FA_ERR_ARG;
+  if (!fa::aligned(K, 8) || !fa::aligned(A, 8) || !fa::aligned(w, 8) || (objective && !fa::aligned(objective, 8)) ||
+      (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::IrlsArgs a{};
+  a.K = K; a.p = p; a.m = m; a.iters = 1; a.lambda = lambda; a.start_from_A = first ? 0 : 1;
+  a.A = A; a.w = w; a.obj = objective; a.status = status;
+  return fa::launch_irls(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+int fa_irls(const double* K, int p, int m, double lambda, int iters, double* A_out, float* c_out, double* w_out,
+            double* obj_out, int* status, void* stream) {
+  if (!K || !c_out || p < 1 || p > FA_MAX_P || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda))
+    return FA_ERR_ARG;
+  if (!fa::aligned(K, 8) || (A_out && !fa::aligned(A_out, 8)) || !fa::aligned(c_out, 4) ||
+      (w_out && !fa::aligned(w_out, 8)) || (obj_out && !fa::aligned(obj_out, 8)) || (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::IrlsArgs a{};
+  a.K = K; a.p = p; a.m = m; a.iters = iters; a.lambda = lambda; a.start_from_A = 0;
+  a.A = A_out; a.c = c_out; a.w = w_out; a.obj = obj_out; a.status = status;
+  return fa::launch_irls(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+int fa_combine(const void* G, int dtype, int p, long long n, const float* c, float* out, void* stream) {
+  if (!G || !c || !out || !fa::shape_ok(p, n, dtype)) return FA_ERR_ARG;
+  if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(c, 4) || !fa::aligned(out, 4)) return FA_ERR_ALIGN;
+  return fa::launch_combine(G, dtype, p, n, c, out, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK
+                                                                                                       : FA_ERR_CUDA;
+}
+
+int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lambda, int iters, float* out,
+                 double* A_out, void* ws, size_t ws_bytes, int* status, void* stream) {
+  if (!G || !out || !ws || !fa::shape_ok(p, n, dtype) || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) ||
+      isinf(lambda))
+    return FA_ERR_ARG;
+  if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(out, 4) || (A_out && !fa::aligned(A_out, 8)) ||
+      !fa::aligned(ws, 16) || (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::Workspace w = fa::carve_ws(ws, p, n, dtype);
+  if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
+  int nblocks = 0;
+  if (fa::launch_gram_partials(G, dtype, p, n, w.partials, status, st, &nblocks) != cudaSuccess) return FA_ERR_CUDA;
+  fa::IrlsArgs a{};
+  a.partials = w.partials; a.nblocks = nblocks; a.Kbuf = w.Kbuf;
+  a.p = p; a.m = m; a.iters = iters; a.lambda = lambda; a.start_from_A = 0;
+  a.A = A_out; a.c = w.c; a.status = status;
+  if (fa::launch_irls(a, st) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_combine(G, dtype, p, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
+  return FA_OK;
+}
+
+int fa_aggregate_host(const void* G_host, int dtype, int p, long long n, int m, double lambda, int iters,
+                      float* out_host, int* status_host, void* G_dev, float* out_dev, void* ws, size_t ws_bytes,
+                      int* status_dev, void* stream) {
+  if (!G_host || !out_host || !G_dev || !out_dev || !fa::shape_ok(p, n, dtype)) return FA_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t gbytes = (size_t)p * (size_t)n * (dtype == FA_F32 ? 4 : 2);
+  // validate everything else before the first copy is enqueued
+  if (!ws || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda)) return FA_ERR_ARG;
+  if (!fa::aligned(G_dev, dtype == FA_F32 ? 4 : 2) || !fa::aligned(out_dev, 4) || !fa::aligned(ws, 16) ||
+      (status_dev && !fa::aligned(status_dev, 4)))
+    return FA_ERR_ALIGN;
+  if (ws_bytes < fa::carve_ws(ws, p, n, dtype).total) return FA_ERR_WORKSPACE;
+  if (cudaMemcpyAsync(G_dev, G_host, gbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return FA_ERR_CUDA;
+  int rc = fa_aggregate(G_dev, dtype, p, n, m, lambda, iters, out_dev, nullptr, ws, ws_bytes, status_dev, stream);
+  if (rc != FA_OK) return rc;
+  if (cudaMemcpyAsync(out_host, out_dev, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return FA_ERR_CUDA;
+  if (status_host && status_dev &&
+      cudaMemcpyAsync(status_host, status_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return FA_ERR_CUDA;
+  return FA_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Persistent single-block kernel around the p-dimensional IRLS (Algorithm 1, IRLS step): every
+// round -- ratios, Beta-likelihood weights, pairwise regulariser, Jacobi eigensolve -- runs out
+// of shared memory; global memory is touched only to read K and write A, c, w, objective.
+#include "fa_irls_core.cuh"
+#include "fa_kernels.h"
+
+namespace fa {
+
+__global__ void irls_kernel(IrlsArgs a) {
+  extern __shared__ __align__(16) unsigned char irls_smem[];
+  fa_irls::Ctx ctx{(int)threadIdx.x, (int)blockDim.x};
+  const double* K = a.K;
+  if (a.partials) {
+    // sum the Gram pass's per-block triangles in block order into the full symmetric matrix
+    const int p = a.p, ntri = p * (p + 1) / 2;
+    for (int idx = ctx.tid; idx < p * p; idx += ctx.nt) {
+      int i = idx / p, j = idx - i * p;
+      if (j < i) { int t = i; i = j; j = t; }
+      const int c = i * p - (i * (i - 1)) / 2 + (j - i);
+      double sum = 0.0;
+      for (int b = 0; b < a.nblocks; ++b) sum += a.partials[(size_t)b * ntri + c];
+      a.Kbuf[idx] = sum;
+    }
+    __syncthreads();
+    K = a.Kbuf;
+  }
+  fa_irls::Smem s;
+  fa_irls::carve(s, irls_smem, a.p, ctx.nt);
+  fa_irls::Outputs o{a.A, a.c, a.w, a.obj, a.status};
+  const int st = fa_irls::run(ctx, s, K, a.p, a.m, a.lambda, a.iters, a.start_from_A != 0, o);
+  if (st && a.status && ctx.tid == 0) atomicOr(a.status, st);
+}
+
+cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
+  const int nt = a.p <= 16 ? 128 : a.p <= 32 ? 256 : 512;
+  const size_t smem = fa_irls::smem_bytes(a.p, nt);
+  cudaError_t e = cudaFuncSetAttribute(irls_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  irls_kernel<<<1, nt, smem, st>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace fa

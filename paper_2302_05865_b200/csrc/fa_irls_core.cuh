@@ -1,0 +1,463 @@
+// IRLS of the Flag Aggregator carried out in p-dimensional coordinates by ONE thread block.
+//
+// Input is only K (p x p inner products of the gradients).  The n-dimensional problem of
+// Algorithm 1 / Eq. (5) is mapped isometrically to R^r, r = rank(K):
+//   * Kt = D^-1 K D^-1 with D = diag(sqrt(K_ii))  (unit diagonal, so the truncation of null
+//     directions below does not depend on the scale of any single worker);
+//   * Kt = V L V^T by cyclic Jacobi; the r eigenpairs with L_k > RANK_REL * L_1 are kept;
+//   * f_i = L^(1/2) V^T D e_i in R^r satisfies <f_i, f_j> = K_ij, and Q = G D^-1 V L^(-1/2)
+//     (n x r) has orthonormal columns with Q^T g_i = f_i.
+// A subspace Y = Q Z is represented by Z (r x m); in gradient coordinates Y = G A with
+// A = D^-1 V L^(-1/2) Z.  Each round forms T = sum w_i f_i f_i^T + sum w_ij (f_i-f_j)(f_i-f_j)^T
+// = F M F^T, diagonalises it by Jacobi (started in the previous round's eigenbasis, where T is
+// already nearly diagonal), keeps the m leading eigenvectors and evaluates the terms under the
+// square roots of Eq. (5) as squared residual norms, i.e. as sums of squares over the discarded
+// eigen-directions -- no "1 - x" cancellation.
+//
+// The code is written as phases separated by block barriers, every phase a strided loop over
+// independent items, so that it can also be compiled for the host with one "thread" (used to
+// debug the arithmetic without a GPU).
+#pragma once
+
+#include <math.h>
+#include <stdint.h>
+
+#ifndef FA_IRLS_HOST
+#define FA_FN __device__ __forceinline__
+#define FA_HD __host__ __device__ inline
+#else
+#define FA_FN static inline
+#define FA_HD static inline
+#endif
+
+namespace fa_irls {
+
+constexpr double kEps = 1e-6;          // floor on sqrt(term) inside a weight
+constexpr double kZeroNormRel = 1e-30; // K_ii <= this * max K_kk: zero gradient
+constexpr double kSamePairRel = 1e-12; // D_ij^2 <= this * (K_ii + K_jj): identical pair
+constexpr double kRankRel = 1e-12;     // eigenvalue <= this * largest: direction dropped
+constexpr double kJacobiTol = 1e-15;   // rotate while |a_pq| > tol * sqrt(|a_pp a_qq|)
+constexpr int kMaxSweeps = 40;
+constexpr int kMaxP = 64;
+
+constexpr int ST_NONFINITE = 1, ST_RANK0 = 2, ST_RANK_LT_M = 4, ST_EIG_SWEEPS = 8;
+
+struct Ctx {
+  int tid, nt;
+#ifndef FA_IRLS_HOST
+  FA_FN void sync() const { __syncthreads(); }
+#else
+  void sync() const {}
+#endif
+};
+
+// Shared-memory image.  Matrices are (pp x ld) doubles, pp = p rounded up to even, ld odd.
+struct Smem {
+  double *T, *J, *P, *M, *Aacc, *tmp;   // six matrix buffers, rotated by pointer swaps
+  double *kd, *dinv, *fn, *u, *w, *wused, *ev, *red;
+  double *rc, *rs;                       // rotation cos / sin per pair
+  int *ra, *rb, *ord;                    // rotation indices per pair, sort order
+  int *flags;                            // [0],[3] rotated-this-sweep (by sweep parity), [1] scratch
+  int ld;
+};
+
+FA_HD size_t smem_bytes(int p, int nt) {
+  int pp = (p + 1) & ~1;
+  int ld = pp + 1;
+  size_t doubles = (size_t)6 * pp * ld + (size_t)7 * pp + nt + 2 * (pp / 2 + 1);
+  size_t ints = (size_t)2 * (pp / 2 + 1) + pp + 8;
+  return doubles * sizeof(double) + ints * sizeof(int) + 64;
+}
+
+FA_FN void carve(Smem& s, void* base, int p, int nt) {
+  int pp = (p + 1) & ~1;
+  int ld = pp + 1;
+  double* d = reinterpret_cast<double*>(base);
+  s.ld = ld;
+  s.T = d; d += (size_t)pp * ld;
+  s.J = d; d += (size_t)pp * ld;
+  s.P = d; d += (size_t)pp * ld;
+  s.M = d; d += (size_t)pp * ld;
+  s.Aacc = d; d += (size_t)pp * ld;
+  s.tmp = d; d += (size_t)pp * ld;
+  s.kd = d; d += pp; s.dinv = d; d += pp; s.fn = d; d += pp; s.u = d; d += pp;
+  s.w = d; d += pp; s.wused = d; d += pp; s.ev = d; d += pp;
+  s.red = d; d += nt;
+  s.rc = d; d += pp / 2 + 1; s.rs = d; d += pp / 2 + 1;
+  int* q = reinterpret_cast<int*>(d);
+  s.ra = q; q += pp / 2 + 1; s.rb = q; q += pp / 2 + 1; s.ord = q; q += pp; s.flags = q;
+}
+
+// Deterministic block-wide sum; every thread gets the result.
+FA_FN double block_sum(const Ctx& c, const Smem& s, double v) {
+#ifndef FA_IRLS_HOST
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+  c.sync();                                // s.red may still be read from a previous call
+  if ((c.tid & 31) == 0) s.red[c.tid >> 5] = v;
+  c.sync();
+  double tot = 0.0;
+  int nw = (c.nt + 31) >> 5;
+  for (int k = 0; k < nw; ++k) tot += s.red[k];
+  return tot;
+#else
+  (void)c; (void)s;
+  return v;
+#endif
+}
+
+// Cyclic Jacobi with round-robin pairing.  T (dim x dim, symmetric, both halves stored) is
+// driven to diagonal form; J accumulates the rotations (J <- J * R).  Rows/columns dim..pp-1 of
+// T must be zero; they take identity rotations.  Returns the number of sweeps made.
+FA_FN int jacobi(const Ctx& c, const Smem& s, double* T, double* J, int dim, int jrows) {
+  const int ld = s.ld;
+  const int pp = (dim + 1) & ~1;
+  const int np = pp >> 1;
+  if (dim < 2) return 0;
+  int sweep = 0;
+  // "rotated in this sweep" flag, double-buffered by sweep parity (slots 0 and 3) so that
+  // clearing the next sweep's flag cannot race with setting the current one
+  if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
+  c.sync();
+  for (; sweep < kMaxSweeps; ++sweep) {
+    int* rotated = &s.flags[(sweep & 1) ? 3 : 0];
+    if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
+    for (int rd = 0; rd < pp - 1; ++rd) {
+      // phase 1: one thread per pair picks the rotation
+      for (int k = c.tid; k < np; k += c.nt) {
+        int a, b;
+        if (k == 0) { a = pp - 1; b = rd; }
+        else { a = (rd + k) % (pp - 1); b = (rd + (pp - 1) - k) % (pp - 1); }
+        if (a > b) { int t = a; a = b; b = t; }
+        double cs = 1.0, sn = 0.0;
+        if (b < dim) {
+          double app = T[a * ld + a], aqq = T[b * ld + b], apq = T[a * ld + b];
+          double mag = fabs(apq);
+          if (mag > kJacobiTol * sqrt(fabs(app * aqq)) && mag > 1e-290) {
+            double theta = (aqq - app) / (2.0 * apq);
+            double t;
+            if (fabs(theta) > 1e150) t = 0.5 / theta;
+            else {
+              t = 1.0 / (fabs(theta) + sqrt(theta * theta + 1.0));
+              if (theta < 0.0) t = -t;
+            }
+            cs = 1.0 / sqrt(t * t + 1.0);
+            sn = t * cs;
+            *rotated = 1;
+          }
+        }
+        s.ra[k] = a; s.rb[k] = b; s.rc[k] = cs; s.rs[k] = sn;
+      }
+      c.sync();
+      // phase 2: every 2x2 block (pair k rows, pair l columns) takes both rotations at once
+      for (int idx = c.tid; idx < np * np; idx += c.nt) {
+        int k = idx / np, l = idx - k * np;
+        int a = s.ra[k], b = s.rb[k], cc = s.ra[l], d = s.rb[l];
+        double ck = s.rc[k], sk = s.rs[k], cl = s.rc[l], sl = s.rs[l];
+        if (ck == 1.0 && sk == 0.0 && cl == 1.0 && sl == 0.0) continue;
+        double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+        double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+        double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+        double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
+        double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
+        if (k == l) { zad = 0.0; zbc = 0.0; }
+        T[a * ld + cc] = zac; T[a * ld + d] = zad; T[b * ld + cc] = zbc; T[b * ld + d] = zbd;
+      }
+      for (int idx = c.tid; idx < jrows * np; idx += c.nt) {
+        int x = idx / np, k = idx - x * np;
+        double ck = s.rc[k], sk = s.rs[k];
+        if (ck == 1.0 && sk == 0.0) continue;
+        int a = s.ra[k], b = s.rb[k];
+        double va = J[x * ld + a], vb = J[x * ld + b];
+        J[x * ld + a] = ck * va - sk * vb;
+        J[x * ld + b] = sk * va + ck * vb;
+      }
+      c.sync();
+    }
+    int again = *rotated;
+    c.sync();
+    if (!again) { ++sweep; break; }
+  }
+  return sweep;
+}
+
+// ev[k] = T[k][k]; ord[q] = index of the q-th largest (ties by index).  All threads return
+// the number of eigenvalues > kRankRel * largest among the first `limit` in that order.
+FA_FN int sort_eigs(const Ctx& c, const Smem& s, const double* T, int dim, int limit) {
+  const int ld = s.ld;
+  for (int k = c.tid; k < dim; k += c.nt) s.ev[k] = T[k * ld + k];
+  c.sync();
+  for (int k = c.tid; k < dim; k += c.nt) {
+    double e = s.ev[k];
+    int rank = 0;
+    for (int l = 0; l < dim; ++l) {
+      double o = s.ev[l];
+      rank += (o > e || (o == e && l < k)) ? 1 : 0;
+    }
+    s.ord[rank] = k;
+  }
+  c.sync();
+  double top = s.ev[s.ord[0]];
+  int keep = 0;
+  if (top > 0.0) {
+    int lim = limit < dim ? limit : dim;
+    for (int q = 0; q < lim; ++q) keep += (s.ev[s.ord[q]] > kRankRel * top) ? 1 : 0;
+  }
+  return keep;
+}
+
+// From residual coordinates Res (rows k0..r-1 are the part of f_i outside the subspace) and the
+// full coordinates P: u_i, next data weights w_i, the matrix M of the next weighted PCA and the
+// value of Eq. (5).  `uniform` builds the round-one weights instead (u is not needed then).
+FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
+                                   double coef, bool uniform) {
+  const int ld = s.ld;
+  double part = 0.0;
+  for (int i = c.tid; i < p; i += c.nt) {
+    double ui = 0.0, wi = 0.0;
+    if (s.dinv[i] != 0.0) {
+      if (uniform) wi = 1.0;
+      else {
+        double acc = 0.0;
+        for (int k = k0; k < r; ++k) { double v = Res[k * ld + i]; acc += v * v; }
+        ui = acc / s.fn[i];
+        double root = sqrt(ui);
+        part += root;
+        wi = 1.0 / (s.fn[i] * fmax(root, kEps));
+      }
+    }
+    s.u[i] = ui;
+    s.w[i] = wi;
+  }
+  c.sync();
+  if (coef > 0.0) {
+    // off-diagonal entries M_ij = -2 w_ij (ordered pairs: each unordered pair counted twice)
+    for (int idx = c.tid; idx < p * p; idx += c.nt) {
+      int i = idx / p, j = idx - i * p;
+      if (i == j) continue;
+      double d2 = 0.0, res2 = 0.0;
+      for (int k = 0; k < r; ++k) { double v = s.P[k * ld + i] - s.P[k * ld + j]; d2 += v * v; }
+      double wij = 0.0;
+      if (d2 > kSamePairRel * (s.fn[i] + s.fn[j])) {
+        if (uniform) wij = coef;
+        else {
+          for (int k = k0; k < r; ++k) { double v = Res[k * ld + i] - Res[k * ld + j]; res2 += v * v; }
+          double root = sqrt(res2 / d2);
+          part += coef * root;
+          wij = coef / (d2 * fmax(root, kEps));
+        }
+      }
+      s.M[i * ld + j] = -2.0 * wij;
+    }
+    c.sync();
+    for (int i = c.tid; i < p; i += c.nt) {
+      double acc = 0.0;
+      for (int j = 0; j < p; ++j) if (j != i) acc -= s.M[i * ld + j];
+      s.M[i * ld + i] = s.w[i] + acc;
+    }
+  }
+  double obj = block_sum(c, s, part);   // contains the barriers that publish M and w
+  return obj;
+}
+
+struct Outputs {
+  double* A;          // p x m or null
+  float* c;           // p or null
+  double* w;          // p or null
+  double* obj;        // iters (or 1) or null
+  int* status;        // or null
+};
+
+FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int iters) {
+  for (int i = c.tid; i < p * m; i += c.nt) if (o.A) o.A[i] = 0.0;
+  for (int i = c.tid; i < p; i += c.nt) { if (o.c) o.c[i] = 0.f; if (o.w) o.w[i] = 0.0; }
+  for (int i = c.tid; i < iters; i += c.nt) if (o.obj) o.obj[i] = 0.0;
+}
+
+// K: p x p inner products (global or shared memory).  start_from_A: take the subspace in o.A as
+// the current one for the first reweighting (single-step interface); otherwise round one is
+// uniform.  Returns the status bits (same value in every thread).
+FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, int iters,
+              bool start_from_A, const Outputs& o) {
+  const int ld = s.ld;
+  const int pp = (p + 1) & ~1;
+  int status = 0;
+
+  // ---- load K, reject non-finite input
+  if (c.tid == 0) { s.flags[1] = 0; }
+  c.sync();
+  for (int idx = c.tid; idx < pp * ld; idx += c.nt) { s.T[idx] = 0.0; s.J[idx] = 0.0; s.Aacc[idx] = 0.0; s.P[idx] = 0.0; s.M[idx] = 0.0; s.tmp[idx] = 0.0; }
+  c.sync();
+  for (int idx = c.tid; idx < p * p; idx += c.nt) {
+    int i = idx / p, j = idx - i * p;
+    double v = K[idx];
+    if (!(fabs(v) <= 1.7e308)) s.flags[1] = 1;
+    s.T[i * ld + j] = v;
+  }
+  c.sync();
+  if (s.flags[1]) {
+    write_zero_outputs(c, o, p, m, iters);
+    return ST_NONFINITE;
+  }
+  for (int i = c.tid; i < p; i += c.nt) s.kd[i] = s.T[i * ld + i];
+  c.sync();
+  double kmax = 0.0;
+  for (int i = 0; i < p; ++i) kmax = fmax(kmax, s.kd[i]);
+  if (!(kmax > 0.0)) {
+    write_zero_outputs(c, o, p, m, iters);
+    return ST_RANK0;
+  }
+  for (int i = c.tid; i < p; i += c.nt)
+    s.dinv[i] = (s.kd[i] <= kZeroNormRel * kmax) ? 0.0 : 1.0 / sqrt(s.kd[i]);
+  c.sync();
+
+  // ---- Kt = D^-1 K D^-1 (symmetrised), J = I, eigen-decomposition
+  for (int idx = c.tid; idx < p * p; idx += c.nt) {
+    int i = idx / p, j = idx - i * p;
+    if (j < i) continue;
+    double v = (i == j) ? (s.dinv[i] != 0.0 ? 1.0 : 0.0)
+                        : 0.5 * (s.T[i * ld + j] + s.T[j * ld + i]) * s.dinv[i] * s.dinv[j];
+    s.tmp[i * ld + j] = v; s.tmp[j * ld + i] = v;
+  }
+  for (int i = c.tid; i < p; i += c.nt) s.J[i * ld + i] = 1.0;
+  c.sync();
+  { double* t = s.T; s.T = s.tmp; s.tmp = t; }
+  int sw = jacobi(c, s, s.T, s.J, p, p);
+  if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
+  const int r = sort_eigs(c, s, s.T, p, p);      // rank of the embedding (>= 1 here)
+
+  // ---- P = F (r x p), Aacc = D^-1 V L^(-1/2) (p x r); f-norms
+  for (int idx = c.tid; idx < r * p; idx += c.nt) {
+    int k = idx / p, i = idx - k * p;
+    int col = s.ord[k];
+    double root = sqrt(s.ev[col]);
+    double v = s.J[i * ld + col];
+    s.P[k * ld + i] = (s.dinv[i] != 0.0) ? root * v / s.dinv[i] : 0.0;
+    s.Aacc[i * ld + k] = s.dinv[i] * v / root;
+  }
+  c.sync();
+  for (int i = c.tid; i < p; i += c.nt) {
+    double acc = 0.0;
+    for (int k = 0; k < r; ++k) { double v = s.P[k * ld + i]; acc += v * v; }
+    s.fn[i] = acc;
+  }
+  c.sync();
+
+  const double coef = (lambda > 0.0 && p > 1) ? lambda / (double)(p - 1) : 0.0;
+
+  // ---- weights of the first round
+  if (!start_from_A) {
+    (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true);
+  } else {
+    // Z0 = F A (r x m) -> J buffer; C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
+    for (int idx = c.tid; idx < r * m; idx += c.nt) {
+      int k = idx / m, q = idx - k * m;
+      double acc = 0.0;
+      for (int i = 0; i < p; ++i) acc += s.P[k * ld + i] * o.A[i * m + q];
+      s.J[k * ld + q] = acc;
+    }
+    c.sync();
+    for (int idx = c.tid; idx < m * p; idx += c.nt) {
+      int q = idx / p, i = idx - q * p;
+      double acc = 0.0;
+      for (int k = 0; k < r; ++k) acc += s.J[k * ld + q] * s.P[k * ld + i];
+      s.T[q * ld + i] = acc;
+    }
+    c.sync();
+    for (int idx = c.tid; idx < r * p; idx += c.nt) {
+      int k = idx / p, i = idx - k * p;
+      double acc = s.P[k * ld + i];
+      for (int q = 0; q < m; ++q) acc -= s.J[k * ld + q] * s.T[q * ld + i];
+      s.tmp[k * ld + i] = acc;
+    }
+    c.sync();
+    (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false);
+  }
+
+  int m_eff = 0;
+  for (int t = 0; t < iters; ++t) {
+    for (int i = c.tid; i < p; i += c.nt) s.wused[i] = s.w[i];
+    // ---- T = P M P^T (current basis)
+    if (coef > 0.0) {
+      for (int idx = c.tid; idx < p * r; idx += c.nt) {       // tmp[i][a] = sum_j M[i][j] P[a][j]
+        int i = idx / r, a = idx - i * r;
+        double acc = 0.0;
+        for (int j = 0; j < p; ++j) acc += s.M[i * ld + j] * s.P[a * ld + j];
+        s.tmp[i * ld + a] = acc;
+      }
+      c.sync();
+      for (int idx = c.tid; idx < r * r; idx += c.nt) {
+        int a = idx / r, b = idx - a * r;
+        if (b < a) continue;
+        double acc = 0.0;
+        for (int i = 0; i < p; ++i) acc += s.P[a * ld + i] * s.tmp[i * ld + b];
+        s.T[a * ld + b] = acc; s.T[b * ld + a] = acc;
+      }
+    } else {
+      for (int idx = c.tid; idx < r * r; idx += c.nt) {
+        int a = idx / r, b = idx - a * r;
+        if (b < a) continue;
+        double acc = 0.0;
+        for (int i = 0; i < p; ++i) acc += s.w[i] * s.P[a * ld + i] * s.P[b * ld + i];
+        s.T[a * ld + b] = acc; s.T[b * ld + a] = acc;
+      }
+    }
+    for (int idx = c.tid; idx < pp * pp; idx += c.nt) {
+      int a = idx / pp, b = idx - a * pp;
+      s.J[a * ld + b] = (a == b) ? 1.0 : 0.0;
+      if (a >= r || b >= r) s.T[a * ld + b] = 0.0;
+    }
+    c.sync();
+    sw = jacobi(c, s, s.T, s.J, r, r);
+    if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
+    m_eff = sort_eigs(c, s, s.T, r, m);
+
+    // ---- rotate into the new (sorted) eigenbasis: P <- J^T P, Aacc <- Aacc J
+    for (int idx = c.tid; idx < r * p; idx += c.nt) {
+      int k = idx / p, i = idx - k * p;
+      int col = s.ord[k];
+      double acc = 0.0;
+      for (int l = 0; l < r; ++l) acc += s.J[l * ld + col] * s.P[l * ld + i];
+      s.tmp[k * ld + i] = acc;
+    }
+    for (int idx = c.tid; idx < p * r; idx += c.nt) {
+      int i = idx / r, k = idx - i * r;
+      int col = s.ord[k];
+      double acc = 0.0;
+      for (int l = 0; l < r; ++l) acc += s.Aacc[i * ld + l] * s.J[l * ld + col];
+      s.M[i * ld + k] = acc;
+    }
+    c.sync();
+    { double* x = s.P; s.P = s.tmp; s.tmp = x; }
+    { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
+
+    // ---- terms of Eq. (5) at the new subspace, and the next round's weights
+    double obj = weights_and_objective(c, s, s.P, m_eff, r, p, coef, false);
+    if (o.obj && c.tid == 0) o.obj[t] = obj;
+  }
+  if (m_eff < m) status |= ST_RANK_LT_M;
+
+  // ---- outputs
+  if (o.A) {
+    for (int idx = c.tid; idx < p * m; idx += c.nt) {
+      int i = idx / m, q = idx - i * m;
+      o.A[idx] = (q < m_eff) ? s.Aacc[i * ld + q] : 0.0;
+    }
+  }
+  if (o.w) for (int i = c.tid; i < p; i += c.nt) o.w[i] = s.wused[i];
+  if (o.c) {
+    for (int k = c.tid; k < m_eff; k += c.nt) {        // s_k = sum_j P[k][j]  (Z^T F 1)
+      double acc = 0.0;
+      for (int j = 0; j < p; ++j) acc += s.P[k * ld + j];
+      s.ev[k] = acc;
+    }
+    c.sync();
+    for (int i = c.tid; i < p; i += c.nt) {
+      double acc = 0.0;
+      for (int k = 0; k < m_eff; ++k) acc += s.Aacc[i * ld + k] * s.ev[k];
+      o.c[i] = (float)(acc / (double)p);
+    }
+  }
+  return status;
+}
+
+}  // namespace fa_irls

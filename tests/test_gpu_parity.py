@@ -1,0 +1,225 @@
+"""CUDA path vs the CPU oracle, through the C ABI (python binding = argument marshalling only).
+
+Tolerances (floating point): aggregate relative L2 <= 1e-4 and principal angles < 1e-3 rad for
+fp32 gradients, 2e-3 and 1e-2 rad for bf16 gradients.  Inner products: |K - K_oracle| <=
+5e-7 * sqrt(K_ii K_jj) (fp32 products, fp32 runs of <= 64 columns, fp64 above that).
+"""
+import numpy as np
+import pytest
+import torch
+
+import synthetic_inputs as si
+from oracle import fa_oracle as fo
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"f32": (1e-4, 1e-3), "bf16": (2e-3, 1e-2)}
+GRAM_TOL = 5e-7
+
+
+@pytest.fixture(scope="module")
+def fa():
+    import paper_2302_05865_b200 as mod
+    return mod
+
+
+def _gram_err(K, Kref):
+    scale = np.sqrt(np.outer(np.diag(Kref), np.diag(Kref)))
+    scale[scale == 0] = 1.0
+    return float(np.max(np.abs(K - Kref) / scale))
+
+
+LADDER = [
+    # p, n, kind, bf16, misalign
+    (1, 1, "gauss", False, 0), (2, 3, "gauss", False, 1), (3, 5, "noisy_mean", False, 0),
+    (4, 31, "noisy_mean", False, 3), (7, 33, "dup_zero", False, 1), (8, 1023, "gauss", False, 2),
+    (12, 4097, "noisy_mean", False, 0), (15, 65_537, "noisy_mean", False, 1), (15, 300_002, "dup_zero", False, 0),
+    (16, 70_000, "gauss", False, 0), (17, 40_001, "noisy_mean", False, 0), (31, 50_000, "dup_zero", False, 2),
+    (32, 9_999, "gauss", False, 1), (33, 20_000, "noisy_mean", False, 0), (63, 30_001, "noisy_mean", False, 0),
+    (64, 12_345, "gauss", False, 3),
+    (5, 7, "gauss", True, 1), (15, 100_003, "noisy_mean", True, 0), (16, 50_000, "dup_zero", True, 4),
+    (31, 40_002, "noisy_mean", True, 2), (63, 66_000, "dup_zero", True, 0), (64, 8_191, "gauss", True, 5),
+]
+
+
+@pytest.mark.parametrize("p,n,kind,bf16,mis", LADDER)
+def test_gram_matches_plain_inner_products(fa, p, n, kind, bf16, mis):
+    from tests.gpu_util import to_device, redzones_intact
+    G_np = si.ladder_case(p, n, 11, kind, bf16=bf16)
+    G, buf = to_device(G_np, misalign_elems=mis)
+    K = fa.fa_gram(G)
+    K2 = fa.fa_gram(G)
+    torch.cuda.synchronize()
+    assert torch.equal(K, K2)                                   # fixed reduction order
+    Kref = fo.inner_products(si.to_float64(G_np))
+    Kh = K.cpu().numpy()
+    assert np.array_equal(Kh, Kh.T)
+    assert _gram_err(Kh, Kref) < GRAM_TOL
+    assert redzones_intact(buf, 64 + mis, p * n)
+    if kind == "dup_zero" and p >= 3:                           # identical rows give identical entries
+        assert Kh[0, 0] == Kh[0, 1] == Kh[1, 1]
+        assert not Kh[p - 1].any()
+
+
+@pytest.mark.parametrize("p,n,kind,bf16,mis", [c for c in LADDER if c[1] > 1])
+def test_combine_matches_weighted_row_sum(fa, p, n, kind, bf16, mis):
+    from tests.gpu_util import to_device
+    G_np = si.ladder_case(p, n, 12, kind, bf16=bf16)
+    G, _ = to_device(G_np, misalign_elems=mis)
+    c = np.random.default_rng(p * 1000 + n).standard_normal(p).astype(np.float32)
+    guard = torch.full((n + 128,), float("nan"), device="cuda")
+    out = guard[64 + (mis % 4):64 + (mis % 4) + n]
+    fa.fa_combine(G, torch.from_numpy(c).cuda(), out=out)
+    torch.cuda.synchronize()
+    ref = c.astype(np.float64) @ si.to_float64(G_np)
+    scale = np.abs(c.astype(np.float64)) @ np.abs(si.to_float64(G_np)) + 1e-30
+    assert np.max(np.abs(out.cpu().numpy() - ref) / scale) < 1e-5
+    assert torch.isnan(guard[:64 + (mis % 4)]).all() and torch.isnan(guard[64 + (mis % 4) + n:]).all()
+
+
+IRLS_CASES = [
+    (1, 9, "noisy_mean", 1, 0.0, 3), (2, 5, "noisy_mean", 1, 0.3, 4), (3, 33, "dup_zero", 2, 0.2, 5),
+    (7, 33, "dup_zero", 3, 0.0, 6), (15, 2000, "noisy_mean", 8, 0.01, 10), (16, 100, "gauss", 8, 0.1, 6),
+    (17, 64, "noisy_mean", 9, 0.05, 6), (31, 3000, "noisy_mean", 12, 0.01, 12), (6, 3, "gauss", 4, 0.1, 5),
+    (63, 200, "dup_zero", 16, 0.02, 8), (64, 300, "noisy_mean", 20, 0.01, 8),
+]
+
+
+@pytest.mark.parametrize("p,n,kind,m,lam,iters", IRLS_CASES)
+def test_irls_rounds_match_oracle_from_exact_inner_products(fa, p, n, kind, m, lam, iters):
+    """K comes from the oracle's plain definition; only the p-dimensional IRLS kernel is on trial."""
+    G = si.ladder_case(p, n, 5, kind).astype(np.float64)
+    ref = fo.fa_aggregate(G, m, lam, iters)
+    K = torch.from_numpy(fo.inner_products(G)).cuda()
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    w = torch.zeros(p, dtype=torch.float64, device="cuda")
+    obj = torch.zeros(iters, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = fa.fa_irls(K, m, lam, iters, A_out=A, w_out=w, obj_out=obj, status=status)
+    torch.cuda.synchronize()
+    k = ref["Y"].shape[1]
+    st = int(status.item())
+    assert st & ~fa.ST_RANK_LT_M == 0 and bool(st & fa.ST_RANK_LT_M) == (k < m)
+    Ah = A.cpu().numpy()
+    assert not Ah[:, k:].any()
+    Y = G.T @ Ah[:, :k]
+    assert np.abs(Y.T @ Y - np.eye(k)).max() < 1e-9
+    if k:
+        assert fo.principal_angles(ref["Y"], Y).max() < 1e-7
+    assert np.allclose(obj.cpu().numpy(), ref["objective"], rtol=0, atol=1e-9)
+    assert np.allclose(w.cpu().numpy(), ref["w"], rtol=1e-6, atol=0)
+    d = c.cpu().numpy().astype(np.float64) @ G
+    assert fo.rel_l2(d, ref["d"]) < 1e-6
+
+    # the single-round entry point, iterated, walks the same path
+    A1 = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    o1 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    objs = []
+    for t in range(iters):
+        fa.fa_irls_step(K, m, lam, t == 0, A1, objective=o1)
+        objs.append(float(o1.item()))
+    assert np.allclose(objs, ref["objective"], rtol=0, atol=1e-9)
+    if k:
+        assert fo.principal_angles(ref["Y"], G.T @ A1.cpu().numpy()[:, :k]).max() < 1e-7
+
+
+def _aggregate_and_compare(fa, G_np, m, lam, iters, dtype_key, mis=0):
+    from tests.gpu_util import to_device, redzones_intact, subspace_from_A
+    p, n = G_np.shape
+    G, buf = to_device(G_np, misalign_elems=mis)
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    guard = torch.full((n + 128,), float("nan"), device="cuda")
+    out = guard[64:64 + n]
+    fa.fa_aggregate(G, m, lam, iters, out=out, A_out=A, status=status)
+    out2 = fa.fa_aggregate(G, m, lam, iters)
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    assert redzones_intact(buf, 64 + mis, p * n)
+    assert torch.isnan(guard[:64]).all() and torch.isnan(guard[64 + n:]).all()
+    X = si.to_float64(G_np)
+    ref = fo.fa_aggregate(X, m, lam, iters)
+    k = ref["Y"].shape[1]
+    st = int(status.item())
+    assert st & ~fa.ST_RANK_LT_M == 0, f"device status {st}"
+    rel_tol, ang_tol = TOL[dtype_key]
+    rel = fo.rel_l2(out.cpu().numpy(), ref["d"])
+    Y = subspace_from_A(G_np, A.cpu().numpy())
+    assert Y.shape[1] == k
+    ang = float(fo.principal_angles(ref["Y"], Y).max()) if k else 0.0
+    assert rel < rel_tol, f"relative L2 {rel}"
+    assert ang < ang_tol, f"principal angle {ang}"
+    return rel, ang
+
+
+AGG_LADDER = [
+    (1, 17, "noisy_mean", False, 1, 0.0, 3, 0), (2, 3, "gauss", False, 1, 0.5, 4, 1),
+    (3, 5, "noisy_mean", False, 2, 0.1, 5, 0), (7, 33, "dup_zero", False, 3, 0.2, 6, 1),
+    (15, 65_537, "noisy_mean", False, 8, 0.01, 10, 1), (16, 70_000, "gauss", False, 8, 0.1, 6, 0),
+    (17, 40_001, "noisy_mean", False, 9, 0.05, 6, 0), (31, 50_000, "dup_zero", False, 12, 0.01, 8, 2),
+    (33, 20_000, "noisy_mean", False, 12, 0.0, 6, 0), (64, 12_345, "noisy_mean", False, 20, 0.01, 6, 3),
+    (15, 100_003, "noisy_mean", True, 8, 0.01, 8, 0), (31, 40_002, "noisy_mean", True, 12, 0.02, 8, 2),
+    (63, 66_000, "dup_zero", True, 16, 0.01, 8, 0),
+]
+
+
+@pytest.mark.parametrize("p,n,kind,bf16,m,lam,iters,mis", AGG_LADDER)
+def test_aggregate_matches_oracle_on_the_ladder(fa, p, n, kind, bf16, m, lam, iters, mis):
+    G_np = si.ladder_case(p, n, 21, kind, bf16=bf16)
+    _aggregate_and_compare(fa, G_np, m, lam, iters, "bf16" if bf16 else "f32", mis)
+
+
+@pytest.mark.parametrize("name,n", [("cfg1", None), ("cfg2", 1_300_003), ("cfg3", 700_001),
+                                    ("cfg4", 2_000_000), ("cfg5", 400_000)])
+def test_aggregate_matches_oracle_on_the_workload_recipes(fa, name, n):
+    w = si.WORKLOADS[name]
+    if n is not None:
+        w = w.scaled(n)
+    G_np = si.generate(w)
+    _aggregate_and_compare(fa, G_np, w.m, w.lam, w.iters, w.dtype)
+
+
+def test_degenerate_inputs_report_status_and_stay_finite(fa):
+    G = torch.zeros((5, 1000), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    A = torch.ones((5, 2), dtype=torch.float64, device="cuda")
+    out = fa.fa_aggregate(G, 2, 0.1, 3, A_out=A, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == fa.ST_RANK0 and not out.any() and not A.any()
+    G = torch.randn((5, 1000), device="cuda")
+    G[2, 17] = float("inf")
+    out = fa.fa_aggregate(G, 2, 0.1, 3, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == fa.ST_NONFINITE and not out.any()
+
+
+def test_host_side_argument_checks(fa):
+    G = torch.randn((4, 100), device="cuda")
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate(G, 5, 0.0, 3)                 # m > p
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate(G, 2, -1.0, 3)                # negative lambda
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate(G, 2, float("nan"), 3)
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate(G, 2, 0.0, 0)                 # no rounds
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate(G, 2, 0.0, 3, ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(fa.FaError):
+        fa.fa_gram(torch.randn((65, 10), device="cuda"))
+
+
+def test_host_buffer_entry_point_round_trips(fa):
+    w = si.WORKLOADS["cfg1"]
+    G_np = si.generate(w)
+    Gh = torch.from_numpy(G_np).pin_memory()
+    outh = torch.empty(w.n, dtype=torch.float32).pin_memory()
+    sth = torch.zeros(1, dtype=torch.int32).pin_memory()
+    Gd = torch.empty((w.p, w.n), device="cuda")
+    outd = torch.empty(w.n, device="cuda")
+    std = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = fa.new_workspace(Gd, w.m)
+    fa.fa_aggregate_host(Gh, w.m, w.lam, w.iters, outh, Gd, outd, ws, sth, std)
+    torch.cuda.synchronize()
+    ref = fa.fa_aggregate(torch.from_numpy(G_np).cuda(), w.m, w.lam, w.iters)
+    assert torch.equal(outh.cuda(), ref) and int(sth.item()) == 0
