@@ -92,6 +92,12 @@ class ClockSampler:
         return out
 
 
+def whole_job_rate(elapsed_ms_max_over_ranks: float, steps: int, world: int) -> float:
+    """Aggregations per second of the whole job: every rank ran `steps` independent aggregations and the
+    job is as slow as its slowest rank."""
+    return world * steps / (elapsed_ms_max_over_ranks * 1e-3)
+
+
 def oracle_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -220,7 +226,7 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         elapsed_ms = float(t.item())
     ms_per_step = elapsed_ms / args.steps
-    value = world * 1e3 / ms_per_step
+    value = whole_job_rate(elapsed_ms, args.steps, world)
 
     # ---- per-kernel times, same buffers and stream, CUDA events around single launches
     def time_call(fn, reps):
