@@ -47,6 +47,7 @@ extern "C" {
 #define FA_ERR_ALIGN     -2    /* a pointer is not aligned to its element type (K, A: 8 bytes; ws: 16) */
 #define FA_ERR_WORKSPACE -3    /* ws_bytes smaller than fa_workspace_bytes() */
 #define FA_ERR_CUDA      -4    /* a launch failed; cudaGetLastError() has the reason */
+#define FA_ERR_STATIC_LIMIT -5 /* fa_gram_static: shape needs more than the built-in scratch array holds */
 
 /* bits of the device status word */
 #define FA_ST_NONFINITE     1  /* NaN/Inf among the inner products; outputs are zero */
@@ -113,6 +114,28 @@ int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lam
 int fa_aggregate_host(const void* G_host, int dtype, int p, long long n, int m, double lambda,
                       int iters, float* out_host, int* status_host, void* G_dev, float* out_dev,
                       void* ws, size_t ws_bytes, int* status_dev, void* stream);
+
+/* The Gram pass without a workspace argument, for callers that have no device memory to offer
+ * and cannot allocate any: code inside a communication callback, a plugin that only receives its
+ * input and output buffers, a process whose device memory is wholly owned by another runtime's
+ * pool, or a place where cudaMalloc's implicit device synchronisation is not acceptable.  (The
+ * paper has no counterpart; this is a property of the library, not of the method.)
+ *
+ * Same result as fa_gram.  The per-block partial sums go to an array compiled into the library
+ * (FA_STATIC_MAX_BLOCKS * FA_STATIC_MAX_P*(FA_STATIC_MAX_P+1)/2 doubles = 675,840 bytes), which
+ * every GPU that loads the library holds until the process exits.  Limits: p <= FA_STATIC_MAX_P
+ * and a launch of at most FA_STATIC_MAX_BLOCKS blocks (one per SM); anything larger returns
+ * FA_ERR_STATIC_LIMIT and enqueues nothing.  The call allocates and frees nothing.
+ *
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * two calls that can overlap on the GPU (different streams without an ordering between them)
+ * race on it and both results are undefined.  Calls ordered on one stream are fine, and nothing
+ * needs clearing between them: each call overwrites every slot it later reads.
+ *   G : p x n worker-major on the device;  K : out, p x p fp64 on the device */
+#define FA_STATIC_MAX_P      32
+#define FA_STATIC_MAX_BLOCKS 160
+int fa_gram_static(const void* G, int dtype, int p, long long n, double* K, void* stream);
 
 /* Static text for a host return code. */
 const char* fa_error_string(int code);

@@ -35,6 +35,8 @@ _lib.fa_irls.argtypes = [_vp, _i, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_combine.argtypes = [_vp, _i, _i, _ll, _vp, _vp, _vp]
 _lib.fa_aggregate.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_aggregate_host.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.fa_gram_static.argtypes = [_vp, _i, _i, _ll, _vp, _vp]
+_lib.fa_gram_static.restype = _i
 for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_combine", "fa_aggregate",
               "fa_aggregate_host"):
     getattr(_lib, _name).restype = _i
@@ -96,6 +98,17 @@ def fa_gram(G, K=None, ws=None, stream=None):
     ws = new_workspace(G) if ws is None else ws
     _check(_lib.fa_gram(G.data_ptr(), code, p, n, _dev(K, torch.float64, p * p, "K"), ws.data_ptr(),
                         ws.numel() * ws.element_size(), _stream(stream)), "fa_gram")
+    return K
+
+
+def fa_gram_static(G, K=None, stream=None):
+    """fa_gram for callers that cannot allocate: no workspace argument, the partial sums use an array
+    built into the library (p <= 32).  Pass K to keep this wrapper from allocating the result too.
+    Calls that may overlap on the GPU must not share a device: they race on that array."""
+    code, p, n = _gradients(G)
+    K = torch.empty((p, p), dtype=torch.float64, device=G.device) if K is None else K
+    _check(_lib.fa_gram_static(G.data_ptr(), code, p, n, _dev(K, torch.float64, p * p, "K"), _stream(stream)),
+           "fa_gram_static")
     return K
 
 

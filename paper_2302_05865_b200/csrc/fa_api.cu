@@ -64,6 +64,7 @@ const char* fa_error_string(int code) {
     case FA_ERR_ALIGN: return "misaligned pointer";
     case FA_ERR_WORKSPACE: return "workspace too small";
     case FA_ERR_CUDA: return "CUDA launch failed";
+    case FA_ERR_STATIC_LIMIT: return "shape exceeds the built-in scratch array of fa_gram_static (p <= 32, <= 160 blocks)";
     default: return "unknown error code";
   }
 }
