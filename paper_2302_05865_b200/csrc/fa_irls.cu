@@ -6,7 +6,8 @@
 
 namespace fa {
 
-__global__ void irls_kernel(IrlsArgs a) {
+template <int NT>
+__global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   extern __shared__ __align__(16) unsigned char irls_smem[];
   fa_irls::Ctx ctx{(int)threadIdx.x, (int)blockDim.x};
   const double* K = a.K;
@@ -31,13 +32,21 @@ __global__ void irls_kernel(IrlsArgs a) {
   if (st && a.status && ctx.tid == 0) atomicOr(a.status, st);
 }
 
-cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
-  const int nt = a.p <= 16 ? 128 : a.p <= 32 ? 256 : 512;
-  const size_t smem = fa_irls::smem_bytes(a.p, nt);
-  cudaError_t e = cudaFuncSetAttribute(irls_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+template <int NT>
+static cudaError_t launch_nt(const IrlsArgs& a, cudaStream_t st) {
+  const size_t smem = fa_irls::smem_bytes(a.p, NT);
+  cudaError_t e = cudaFuncSetAttribute(irls_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  irls_kernel<<<1, nt, smem, st>>>(a);
+  irls_kernel<NT><<<1, NT, smem, st>>>(a);
   return cudaGetLastError();
+}
+
+// One thread per Jacobi work item where the block size allows it: (p/2)^2 2x2 blocks plus
+// p * p/2 eigenvector row pairs.
+cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
+  if (a.p <= 16) return launch_nt<192>(a, st);
+  if (a.p <= 32) return launch_nt<768>(a, st);
+  return launch_nt<1024>(a, st);
 }
 
 }  // namespace fa

@@ -30,13 +30,20 @@
 #define FA_HD static inline
 #endif
 
+#ifndef FA_IRLS_HOST
+#define FA_RSQRT(x) rsqrt(x)
+#else
+#define FA_RSQRT(x) (1.0 / sqrt(x))
+#endif
+
 namespace fa_irls {
 
 constexpr double kEps = 1e-6;          // floor on sqrt(term) inside a weight
 constexpr double kZeroNormRel = 1e-30; // K_ii <= this * max K_kk: zero gradient
 constexpr double kSamePairRel = 1e-12; // D_ij^2 <= this * (K_ii + K_jj): identical pair
 constexpr double kRankRel = 1e-12;     // eigenvalue <= this * largest: direction dropped
-constexpr double kJacobiTol = 1e-15;   // rotate while |a_pq| > tol * sqrt(|a_pp a_qq|)
+constexpr double kJacobiTol = 1e-17;   // rotate when |a_pq| > tol * sqrt(|a_pp a_qq|)
+constexpr double kJacobiBig = 1e-8;    // sweep again while some rotated |a_pq| exceeded this (relative)
 constexpr int kMaxSweeps = 40;
 constexpr int kMaxP = 64;
 
@@ -105,78 +112,146 @@ FA_FN double block_sum(const Ctx& c, const Smem& s, double v) {
 #endif
 }
 
-// Cyclic Jacobi with round-robin pairing.  T (dim x dim, symmetric, both halves stored) is
-// driven to diagonal form; J accumulates the rotations (J <- J * R).  Rows/columns dim..pp-1 of
-// T must be zero; they take identity rotations.  Returns the number of sweeps made.
-FA_FN int jacobi(const Ctx& c, const Smem& s, double* T, double* J, int dim, int jrows) {
+// Round-robin pairing: in round rd of a sweep over pp (even) indices, pair k is (a, b), a < b.
+FA_FN void pair_of(int rd, int k, int pp, int& a, int& b) {
+  if (k == 0) { a = pp - 1; b = rd; }
+  else {
+    a = rd + k; if (a >= pp - 1) a -= pp - 1;
+    b = rd + (pp - 1) - k; if (b >= pp - 1) b -= pp - 1;
+  }
+  if (a > b) { int t = a; a = b; b = t; }
+}
+
+// Rotation (cs, sn) that annihilates T[a][b]; identity for padded indices and for entries at
+// rounding level.  Written from the double angle, without division and with two rsqrt:
+//   d = a_qq - a_pp, h = 2 a_pq, cos 2phi = |d| / sqrt(d^2 + h^2),
+//   c = sqrt((1 + cos 2phi) / 2), s = sign(d) * h / (2 c sqrt(d^2 + h^2)).
+// Returns true when the entry was "large" (above kJacobiBig relative to its diagonal).
+FA_FN bool rotation(const double* T, int ld, int a, int b, int dim, double& cs, double& sn) {
+  cs = 1.0; sn = 0.0;
+  if (b >= dim) return false;
+  const double app = T[a * ld + a], aqq = T[b * ld + b], apq = T[a * ld + b];
+  const double m2 = apq * apq, ref2 = fabs(app * aqq);
+  if (!(m2 > (kJacobiTol * kJacobiTol) * ref2 && m2 > 1e-280)) return false;
+  const double d = aqq - app, h = 2.0 * apq;
+  const double rinv = FA_RSQRT(d * d + h * h);
+  const double x = 0.5 + 0.5 * fabs(d) * rinv;          // cos^2 phi, in [1/2, 1]
+  const double cinv = FA_RSQRT(x);
+  cs = x * cinv;
+  sn = 0.5 * h * rinv * cinv;
+  if (d < 0.0) sn = -sn;
+  return m2 > (kJacobiBig * kJacobiBig) * ref2;
+}
+
+// Cyclic Jacobi with round-robin pairing.  T (dim x dim, symmetric, both halves stored, rows and
+// columns dim..pp-1 zero) is driven to diagonal form; J accumulates the rotations (J <- J * R).
+// One barrier per round: every work item recomputes the one or two rotations it needs from the
+// round's input matrix (double-buffered in T / Talt), so no thread waits for another thread's
+// parameters.  A pair is rotated whenever its off-diagonal entry is above rounding level;
+// sweeping stops after the first sweep in which no rotated entry exceeded kJacobiBig relative to
+// its diagonal: that sweep's rotations leave entries of the order of its square (quadratic
+// convergence of the cyclic method), i.e. below rounding level.
+// On return *Tio points at the buffer that holds the diagonalised matrix.  Returns the sweeps made.
+FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double* J, int dim, int jrows) {
   const int ld = s.ld;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
   if (dim < 2) return 0;
+  double* T = *Tio;
+  double* Tn = *Taltio;
+  int sh = 0;
+  while ((1 << sh) < np) ++sh;             // items are indexed (k, l) = (idx >> sh, idx & mask)
+  const int mask = (1 << sh) - 1;
+  const int nblk = np << sh, nrow = jrows << sh;
   int sweep = 0;
-  // "rotated in this sweep" flag, double-buffered by sweep parity (slots 0 and 3) so that
-  // clearing the next sweep's flag cannot race with setting the current one
+  // "large rotation in this sweep" flag, double-buffered by sweep parity (slots 0 and 3)
   if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
   c.sync();
   for (; sweep < kMaxSweeps; ++sweep) {
-    int* rotated = &s.flags[(sweep & 1) ? 3 : 0];
+    int* big = &s.flags[(sweep & 1) ? 3 : 0];
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
-      // phase 1: one thread per pair picks the rotation
-      for (int k = c.tid; k < np; k += c.nt) {
-        int a, b;
-        if (k == 0) { a = pp - 1; b = rd; }
-        else { a = (rd + k) % (pp - 1); b = (rd + (pp - 1) - k) % (pp - 1); }
-        if (a > b) { int t = a; a = b; b = t; }
-        double cs = 1.0, sn = 0.0;
-        if (b < dim) {
-          double app = T[a * ld + a], aqq = T[b * ld + b], apq = T[a * ld + b];
-          double mag = fabs(apq);
-          if (mag > kJacobiTol * sqrt(fabs(app * aqq)) && mag > 1e-290) {
-            double theta = (aqq - app) / (2.0 * apq);
-            double t;
-            if (fabs(theta) > 1e150) t = 0.5 / theta;
-            else {
-              t = 1.0 / (fabs(theta) + sqrt(theta * theta + 1.0));
-              if (theta < 0.0) t = -t;
-            }
-            cs = 1.0 / sqrt(t * t + 1.0);
-            sn = t * cs;
-            *rotated = 1;
-          }
+#ifndef FA_IRLS_HOST
+      // Items are strided by the block size, a multiple of the (power-of-two) pair count, so a
+      // thread always meets the same column pair l: it computes that one rotation per round and
+      // fetches the row pair's rotation from the lane that owns it (lane k of its own warp).
+      const int l = c.tid & mask;
+      int al = 0, bl = 0;
+      double cl = 1.0, sl = 0.0;
+      if (l < np) {
+        pair_of(rd, l, pp, al, bl);
+        const bool bigl = rotation(T, ld, al, bl, dim, cl, sl);
+        if (bigl && c.tid < np) *big = 1;
+      }
+      const int total = nblk + nrow;
+      for (int idx = c.tid; idx < ((total + 31) & ~31); idx += c.nt) {
+        const bool isblk = idx < nblk;
+        const int k = isblk ? (idx >> sh) : 0;
+        const double ck = __shfl_sync(0xffffffffu, cl, k);
+        const double sk = __shfl_sync(0xffffffffu, sl, k);
+        const int a = __shfl_sync(0xffffffffu, al, k);
+        const int b = __shfl_sync(0xffffffffu, bl, k);
+        if (idx >= total || l >= np) continue;
+        if (isblk) {
+          // 2x2 block (pair k rows, pair l columns) takes both rotations at once
+          const double xac = T[a * ld + al], xad = T[a * ld + bl], xbc = T[b * ld + al], xbd = T[b * ld + bl];
+          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+          double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
+          double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
+          if (k == l && sk != 0.0) { zad = 0.0; zbc = 0.0; }
+          Tn[a * ld + al] = zac; Tn[a * ld + bl] = zad; Tn[b * ld + al] = zbc; Tn[b * ld + bl] = zbd;
+        } else if (sl != 0.0) {
+          const int x = (idx - nblk) >> sh;
+          const double va = J[x * ld + al], vb = J[x * ld + bl];
+          J[x * ld + al] = cl * va - sl * vb;
+          J[x * ld + bl] = sl * va + cl * vb;
         }
-        s.ra[k] = a; s.rb[k] = b; s.rc[k] = cs; s.rs[k] = sn;
       }
+#else
+      for (int idx = c.tid; idx < nblk + nrow; idx += c.nt) {
+        if (idx < nblk) {
+          // 2x2 block (pair k rows, pair l columns) takes both rotations at once
+          const int k = idx >> sh, l = idx & mask;
+          if (l >= np) continue;
+          int a, b, cc, d;
+          pair_of(rd, k, pp, a, b);
+          pair_of(rd, l, pp, cc, d);
+          double ck, sk, cl, sl;
+          const bool bigk = rotation(T, ld, a, b, dim, ck, sk);
+          if (k == l) { cl = ck; sl = sk; if (bigk) *big = 1; }
+          else (void)rotation(T, ld, cc, d, dim, cl, sl);
+          const double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+          double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
+          double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
+          if (k == l && sk != 0.0) { zad = 0.0; zbc = 0.0; }
+          Tn[a * ld + cc] = zac; Tn[a * ld + d] = zad; Tn[b * ld + cc] = zbc; Tn[b * ld + d] = zbd;
+        } else {
+          const int q = idx - nblk;
+          const int x = q >> sh, k = q & mask;
+          if (k >= np) continue;
+          int a, b;
+          pair_of(rd, k, pp, a, b);
+          double ck, sk;
+          (void)rotation(T, ld, a, b, dim, ck, sk);
+          if (sk == 0.0) continue;
+          const double va = J[x * ld + a], vb = J[x * ld + b];
+          J[x * ld + a] = ck * va - sk * vb;
+          J[x * ld + b] = sk * va + ck * vb;
+        }
+      }
+#endif
       c.sync();
-      // phase 2: every 2x2 block (pair k rows, pair l columns) takes both rotations at once
-      for (int idx = c.tid; idx < np * np; idx += c.nt) {
-        int k = idx / np, l = idx - k * np;
-        int a = s.ra[k], b = s.rb[k], cc = s.ra[l], d = s.rb[l];
-        double ck = s.rc[k], sk = s.rs[k], cl = s.rc[l], sl = s.rs[l];
-        if (ck == 1.0 && sk == 0.0 && cl == 1.0 && sl == 0.0) continue;
-        double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
-        double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-        double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
-        double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
-        double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
-        if (k == l) { zad = 0.0; zbc = 0.0; }
-        T[a * ld + cc] = zac; T[a * ld + d] = zad; T[b * ld + cc] = zbc; T[b * ld + d] = zbd;
-      }
-      for (int idx = c.tid; idx < jrows * np; idx += c.nt) {
-        int x = idx / np, k = idx - x * np;
-        double ck = s.rc[k], sk = s.rs[k];
-        if (ck == 1.0 && sk == 0.0) continue;
-        int a = s.ra[k], b = s.rb[k];
-        double va = J[x * ld + a], vb = J[x * ld + b];
-        J[x * ld + a] = ck * va - sk * vb;
-        J[x * ld + b] = sk * va + ck * vb;
-      }
-      c.sync();
+      { double* t = T; T = Tn; Tn = t; }
     }
-    int again = *rotated;
+    const int again = *big;
     c.sync();
     if (!again) { ++sweep; break; }
   }
+  *Tio = T;
+  *Taltio = Tn;
   return sweep;
 }
 
@@ -321,7 +396,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   for (int i = c.tid; i < p; i += c.nt) s.J[i * ld + i] = 1.0;
   c.sync();
   { double* t = s.T; s.T = s.tmp; s.tmp = t; }
-  int sw = jacobi(c, s, s.T, s.J, p, p);
+  int sw = jacobi(c, s, &s.T, &s.tmp, s.J, p, p);
   if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
   const int r = sort_eigs(c, s, s.T, p, p);      // rank of the embedding (>= 1 here)
 
@@ -407,7 +482,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       if (a >= r || b >= r) s.T[a * ld + b] = 0.0;
     }
     c.sync();
-    sw = jacobi(c, s, s.T, s.J, r, r);
+    sw = jacobi(c, s, &s.T, &s.tmp, s.J, r, r);
     if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
     m_eff = sort_eigs(c, s, s.T, r, m);
 
