@@ -122,7 +122,7 @@ int fa_aggregate_host(const void* G_host, int dtype, int p, long long n, int m, 
  * paper has no counterpart; this is a property of the library, not of the method.)
  *
  * Same result as fa_gram.  The per-block partial sums go to an array compiled into the library
- * (FA_STATIC_MAX_BLOCKS * FA_STATIC_MAX_P*(FA_STATIC_MAX_P+1)/2 doubles = 675,840 bytes), which
+ * (FA_STATIC_MAX_BLOCKS * FA_STATIC_MAX_P*(FA_STATIC_MAX_P+1)/2 doubles plus a 256-byte counter = 676,096 bytes), which
  * every GPU that loads the library holds until the process exits.  Limits: p <= FA_STATIC_MAX_P
  * and a launch of at most FA_STATIC_MAX_BLOCKS blocks (one per SM); anything larger returns
  * FA_ERR_STATIC_LIMIT and enqueues nothing.  The call allocates and frees nothing.

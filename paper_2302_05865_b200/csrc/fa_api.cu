@@ -29,6 +29,7 @@ struct Workspace {
   double* partials;
   double* Kbuf;
   float* c;
+  unsigned int* counter;
   size_t total;
 };
 
@@ -42,6 +43,8 @@ Workspace carve_ws(void* ws, int p, long long n, int dtype) {
   off += round_up((size_t)p * p * sizeof(double));
   w.c = reinterpret_cast<float*>(base + off);
   off += round_up(FA_MAX_P * sizeof(float));
+  w.counter = reinterpret_cast<unsigned int*>(base + off);
+  off += kAlign;
   w.total = off;
   return w;
 }
@@ -82,9 +85,7 @@ int fa_gram(const void* G, int dtype, int p, long long n, double* K, void* ws, s
   fa::Workspace w = fa::carve_ws(ws, p, n, dtype);
   if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int nblocks = 0;
-  if (fa::launch_gram_partials(G, dtype, p, n, w.partials, nullptr, st, &nblocks) != cudaSuccess) return FA_ERR_CUDA;
-  if (fa::launch_reduce_partials(w.partials, nblocks, p, K, st) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_gram(G, dtype, p, n, w.partials, w.counter, K, nullptr, st) != cudaSuccess) return FA_ERR_CUDA;
   return FA_OK;
 }
 
@@ -132,10 +133,9 @@ int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lam
   if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
-  int nblocks = 0;
-  if (fa::launch_gram_partials(G, dtype, p, n, w.partials, status, st, &nblocks) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_gram(G, dtype, p, n, w.partials, w.counter, w.Kbuf, status, st) != cudaSuccess) return FA_ERR_CUDA;
   fa::IrlsArgs a{};
-  a.partials = w.partials; a.nblocks = nblocks; a.Kbuf = w.Kbuf;
+  a.K = w.Kbuf;
   a.p = p; a.m = m; a.iters = iters; a.lambda = lambda; a.start_from_A = 0;
   a.A = A_out; a.c = w.c; a.status = status;
   if (fa::launch_irls(a, st) != cudaSuccess) return FA_ERR_CUDA;

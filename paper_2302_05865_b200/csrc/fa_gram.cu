@@ -7,8 +7,8 @@
 // 16-byte-aligned start and read back with a per-row byte skew.  Eight consumer warps form the
 // products in fp32 (exact for bf16 inputs, correctly rounded for fp32 inputs), keep fp32 running
 // sums over at most kFlushCols columns, then fold them with a warp butterfly into fp64 lane
-// accumulators.  Block totals are written to a per-block slot of the workspace and summed in
-// block order by a second tiny kernel (or by the IRLS kernel), so the result is bit-reproducible.
+// accumulators.  Block totals go to the workspace; the last block to finish adds them up in a
+// fixed order and writes K, so the result is bit-reproducible and no second launch is needed.
 #include "fa_common.cuh"
 #include "fa_kernels.h"
 
@@ -29,7 +29,9 @@ struct Params {
   int tile_cols;       // columns per tile
   int row_stride;      // bytes between staged rows
   long long num_tiles;
-  double* partials;    // [gridDim.x][p(p+1)/2], canonical upper-triangle order
+  double* partials;    // [p(p+1)/2][gridDim.x]: entry c (canonical upper-triangle order) of block b at c*gridDim.x + b
+  unsigned int* counter;   // blocks finished so far (zero at launch)
+  double* K;           // out: p x p, written by the last block to finish
   int* status;
 };
 
@@ -62,6 +64,40 @@ __device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP 
   for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
 #pragma unroll
   for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
+}
+
+// Called by every thread of a block after it has written its entries of `partials`.  The last
+// block to arrive (atomic counter) adds up all blocks' entries and writes the symmetric K.  Each
+// entry is summed by one warp: lane l takes blocks l, l+32, ... in order, then a fixed shuffle
+// tree -- the order does not depend on which block happens to be last, so K is bit-reproducible.
+__device__ __forceinline__ void finish_gram(const Params& prm, int* smem_flag) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned int done = atomicAdd(prm.counter, 1u);
+    *smem_flag = (done == gridDim.x - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!*smem_flag) return;
+  __threadfence();
+  const int p = prm.p, ntri = p * (p + 1) / 2;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int nb = gridDim.x;
+  for (int c = warp; c < ntri; c += nwarps) {
+    const double* src = prm.partials + (size_t)c * nb;
+    double sum = 0.0;
+    for (int b = lane; b < nb; b += 32) sum += __ldcg(src + b);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) {
+      int i = 0, r = c;
+      while (r >= p - i) { r -= p - i; ++i; }
+      const int j = i + r;
+      prm.K[i * p + j] = sum;
+      prm.K[j * p + i] = sum;
+    }
+  }
+  if (threadIdx.x == 0) *prm.counter = 0u;     // leave the counter ready for the next launch
 }
 
 struct Ring {
@@ -222,8 +258,7 @@ __global__ void __launch_bounds__((CW + 1) * 32, 1) gram_tri_kernel(Params prm) 
   else consume_tri<T, V, PB, CW>(prm, stages, stage_bytes, ring, totals, tid);
   __syncthreads();
 
-  // block total -> this block's slot, canonical triangle order (fixed warp order)
-  double* slot = prm.partials + (size_t)blockIdx.x * (prm.p * (prm.p + 1) / 2);
+  // block total (fixed warp order) -> this block's entries, then the last block forms K
   for (int e = tid; e < NACC; e += kThreads) {
     int i = 0, r = e;
     while (r >= PB - i) { r -= PB - i; ++i; }
@@ -231,9 +266,10 @@ __global__ void __launch_bounds__((CW + 1) * 32, 1) gram_tri_kernel(Params prm) 
     if (j < prm.p) {
       double sum = 0.0;
       for (int w = 0; w < kConsumerWarps; ++w) sum += totals[w * NACCP + e];
-      slot[canon_index(i, j, prm.p)] = sum;
+      prm.partials[(size_t)canon_index(i, j, prm.p) * gridDim.x + blockIdx.x] = sum;
     }
   }
+  finish_gram(prm, ring.abort);
 }
 
 // ---- consumers, 16 < p <= 64: rows are cut into blocks of 16; a work item is the triangle of
@@ -366,7 +402,6 @@ __global__ void __launch_bounds__(kThreads, 1) gram_blocks_kernel(Params prm) {
   else consume_blocks<T, NB>(prm, stages, stage_bytes, ring, totals, rowoff_s, tid);
   __syncthreads();
 
-  double* slot = prm.partials + (size_t)blockIdx.x * (prm.p * (prm.p + 1) / 2);
   for (int idx = tid; idx < W * kItemAcc; idx += kThreads) {
     const int item = idx / kItemAcc, e = idx - item * kItemAcc;
     bool tri; int i0, j0;
@@ -389,21 +424,9 @@ __global__ void __launch_bounds__(kThreads, 1) gram_blocks_kernel(Params prm) {
       const int w = item % kConsumerWarps, q = item / kConsumerWarps;
       sum = totals[(size_t)(w * IPW + q) * kItemAcc + e];
     }
-    slot[canon_index(gi, gj, prm.p)] = sum;
+    prm.partials[(size_t)canon_index(gi, gj, prm.p) * gridDim.x + blockIdx.x] = sum;
   }
-}
-
-// ---- sum the block slots in block order -> full symmetric K
-__global__ void reduce_partials_kernel(const double* partials, int nblocks, int p, double* K) {
-  const int ntri = p * (p + 1) / 2;
-  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < p * p; idx += gridDim.x * blockDim.x) {
-    int i = idx / p, j = idx - i * p;
-    if (j < i) { int t = i; i = j; j = t; }
-    const int c = canon_index(i, j, p);
-    double sum = 0.0;
-    for (int b = 0; b < nblocks; ++b) sum += partials[(size_t)b * ntri + c];
-    K[idx] = sum;
-  }
+  finish_gram(prm, ring.abort);
 }
 
 // ---- host side
@@ -481,8 +504,8 @@ size_t gram_partials_bytes(int p, long long n, int dtype) {
   return (size_t)gram_num_blocks(p, n, dtype) * (size_t)(p * (p + 1) / 2) * sizeof(double);
 }
 
-cudaError_t launch_gram_partials(const void* G, int dtype, int p, long long n, double* partials, int* status,
-                                 cudaStream_t st, int* nblocks_out) {
+cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
+                        double* K, int* status, cudaStream_t st) {
   const gram::Shape sh = gram::pick_shape(p);
   const int S = dtype == 0 ? 4 : 2;
   gram::Params prm{};
@@ -493,20 +516,18 @@ cudaError_t launch_gram_partials(const void* G, int dtype, int p, long long n, d
   prm.row_stride = sh.row_bytes + 16;
   prm.num_tiles = (n + prm.tile_cols - 1) / prm.tile_cols;
   prm.partials = partials;
+  prm.counter = counter;
+  prm.K = K;
   prm.status = status;
   const int grid = gram_num_blocks(p, n, dtype);
-  *nblocks_out = grid;
+  cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
+  if (e != cudaSuccess) return e;
   // two elements per shared load when every row starts on an even element
   const bool even = (n % 2 == 0) && ((reinterpret_cast<uintptr_t>(G) % (2 * S)) == 0);
   const int vec = even ? 2 : 1;
   const size_t smem = gram::smem_bytes(sh);
   if (dtype == 0) return gram::dispatch<float>(sh, vec, prm, grid, smem, st);
   return gram::dispatch<__nv_bfloat16>(sh, vec, prm, grid, smem, st);
-}
-
-cudaError_t launch_reduce_partials(const double* partials, int nblocks, int p, double* K, cudaStream_t st) {
-  gram::reduce_partials_kernel<<<(p * p + 255) / 256, 256, 0, st>>>(partials, nblocks, p, K);
-  return cudaGetLastError();
 }
 
 }  // namespace fa

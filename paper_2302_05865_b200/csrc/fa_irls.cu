@@ -11,20 +11,6 @@ __global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   extern __shared__ __align__(16) unsigned char irls_smem[];
   fa_irls::Ctx ctx{(int)threadIdx.x, (int)blockDim.x};
   const double* K = a.K;
-  if (a.partials) {
-    // sum the Gram pass's per-block triangles in block order into the full symmetric matrix
-    const int p = a.p, ntri = p * (p + 1) / 2;
-    for (int idx = ctx.tid; idx < p * p; idx += ctx.nt) {
-      int i = idx / p, j = idx - i * p;
-      if (j < i) { int t = i; i = j; j = t; }
-      const int c = i * p - (i * (i - 1)) / 2 + (j - i);
-      double sum = 0.0;
-      for (int b = 0; b < a.nblocks; ++b) sum += a.partials[(size_t)b * ntri + c];
-      a.Kbuf[idx] = sum;
-    }
-    __syncthreads();
-    K = a.Kbuf;
-  }
   fa_irls::Smem s;
   fa_irls::carve(s, irls_smem, a.p, ctx.nt);
   fa_irls::Outputs o{a.A, a.c, a.w, a.obj, a.status};

@@ -7,20 +7,16 @@ namespace fa {
 
 int sm_count();   // SMs of the current device (cached per device)
 
-// Gram pass -> per-block partial triangles in `partials` (gram_partials_bytes() bytes).
+// Gram pass.  `partials` (gram_partials_bytes() bytes) and `counter` are scratch; K (p x p) is
+// written by the last block to finish.
 int gram_num_blocks(int p, long long n, int dtype);
 size_t gram_partials_bytes(int p, long long n, int dtype);
-cudaError_t launch_gram_partials(const void* G, int dtype, int p, long long n, double* partials, int* status,
-                                 cudaStream_t st, int* nblocks_out);
-cudaError_t launch_reduce_partials(const double* partials, int nblocks, int p, double* K, cudaStream_t st);
+cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
+                        double* K, int* status, cudaStream_t st);
 
-// Persistent single-block IRLS.  If `partials` is non-null the block first sums the Gram slots
-// into Kbuf (p*p doubles) and uses that; otherwise it reads K.
+// Persistent single-block IRLS on K (p x p).
 struct IrlsArgs {
   const double* K;
-  const double* partials;
-  int nblocks;
-  double* Kbuf;
   int p, m, iters;
   double lambda;
   int start_from_A;

@@ -13,9 +13,9 @@
 
 namespace {
 
-// 160 block slots of at most 32*33/2 partial inner products each: 675,840 bytes.
+// 160 block slots of at most 32*33/2 partial inner products each (675,840 bytes) + a 256-byte counter.
 constexpr size_t kScratchDoubles = (size_t)FA_STATIC_MAX_BLOCKS * (FA_STATIC_MAX_P * (FA_STATIC_MAX_P + 1) / 2);
-static __device__ __align__(256) double g_gram_scratch[kScratchDoubles];
+static __device__ __align__(256) double g_gram_scratch[kScratchDoubles + 32];
 
 // Device address of the array, looked up once per device.  In host code `g_gram_scratch` is only a
 // handle for the runtime; the kernels need the address that cudaGetSymbolAddress returns.
@@ -44,10 +44,10 @@ extern "C" int fa_gram_static(const void* G, int dtype, int p, long long n, doub
   double* scratch = scratch_address(&rc);
   if (!scratch) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int nblocks = 0;
-  // Every block overwrites its whole slot and only the first `nblocks` slots are read back, so
-  // nothing left in the array by an earlier call needs clearing.
-  if (fa::launch_gram_partials(G, dtype, p, n, scratch, nullptr, st, &nblocks) != cudaSuccess) return FA_ERR_CUDA;
-  if (fa::launch_reduce_partials(scratch, nblocks, p, K, st) != cudaSuccess) return FA_ERR_CUDA;
+  // The counter (first 256 bytes) is cleared by a memset node on the stream before the kernel;
+  // every block overwrites all of its partial sums and only those are read back, so nothing else
+  // left in the array by an earlier call needs clearing.
+  unsigned int* counter = reinterpret_cast<unsigned int*>(scratch);
+  if (fa::launch_gram(G, dtype, p, n, scratch + 32, counter, K, nullptr, st) != cudaSuccess) return FA_ERR_CUDA;
   return FA_OK;
 }
