@@ -385,7 +385,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     s.dinv[i] = (s.kd[i] <= kZeroNormRel * kmax) ? 0.0 : 1.0 / sqrt(s.kd[i]);
   c.sync();
 
-  // ---- Kt = D^-1 K D^-1 (symmetrised), J = I, eigen-decomposition
+  // ---- Kt = D^-1 K D^-1 (symmetrised, unit diagonal) -> tmp
   for (int idx = c.tid; idx < p * p; idx += c.nt) {
     int i = idx / p, j = idx - i * p;
     if (j < i) continue;
@@ -393,23 +393,70 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
                         : 0.5 * (s.T[i * ld + j] + s.T[j * ld + i]) * s.dinv[i] * s.dinv[j];
     s.tmp[i * ld + j] = v; s.tmp[j * ld + i] = v;
   }
-  for (int i = c.tid; i < p; i += c.nt) s.J[i * ld + i] = 1.0;
+  // remaining diagonal of the factorisation -> u; "already a pivot" marks -> ord (as flags)
+  for (int i = c.tid; i < p; i += c.nt) { s.u[i] = (s.dinv[i] != 0.0) ? 1.0 : 0.0; s.ord[i] = 0; }
   c.sync();
-  { double* t = s.T; s.T = s.tmp; s.tmp = t; }
-  int sw = jacobi(c, s, &s.T, &s.tmp, s.J, p, p);
-  if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
-  const int r = sort_eigs(c, s, s.T, p, p);      // rank of the embedding (>= 1 here)
 
-  // ---- P = F (r x p), Aacc = D^-1 V L^(-1/2) (p x r); f-norms
-  for (int idx = c.tid; idx < r * p; idx += c.nt) {
-    int k = idx / p, i = idx - k * p;
-    int col = s.ord[k];
-    double root = sqrt(s.ev[col]);
-    double v = s.J[i * ld + col];
-    s.P[k * ld + i] = (s.dinv[i] != 0.0) ? root * v / s.dinv[i] : 0.0;
-    s.Aacc[i * ld + k] = s.dinv[i] * v / root;
+  // ---- Cholesky with complete pivoting, Kt = R^T R, R (r x p) kept in P with the original column
+  // order: column i of R is the image f_i / ||g_i|| of worker i in R^r.  Stops when the largest
+  // remaining diagonal entry is <= kRankRel (the diagonal of Kt is 1), which fixes the rank r.
+  int r = 0;
+  for (int k = 0; k < p; ++k) {
+    int piv = -1;
+    double dmax = kRankRel;
+    for (int j = 0; j < p; ++j) {                 // every thread scans; ties go to the lowest index
+      const double dj = s.u[j];
+      if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
+    }
+    if (piv < 0) break;
+    const double rkk = sqrt(dmax), rinv = 1.0 / rkk;
+    for (int j = c.tid; j < p; j += c.nt) {
+      double v;
+      if (j == piv) v = rkk;
+      else if (s.ord[j] != 0) v = 0.0;
+      else {
+        double acc = s.tmp[piv * ld + j];
+        for (int l = 0; l < k; ++l) acc -= s.P[l * ld + piv] * s.P[l * ld + j];
+        v = acc * rinv;
+      }
+      s.P[k * ld + j] = v;
+    }
+    if (c.tid == 0) s.wused[k] = (double)piv;     // pivot order (exact small integers)
+    c.sync();
+    for (int j = c.tid; j < p; j += c.nt) {
+      if (j == piv) { s.ord[j] = 1; s.u[j] = 0.0; }
+      else if (s.ord[j] == 0) { const double v = s.P[k * ld + j]; s.u[j] = fmax(s.u[j] - v * v, 0.0); }
+    }
+    c.sync();
+    r = k + 1;
+  }
+
+  // ---- U = R11^-1 (R11 = pivot columns of R, upper triangular) by back substitution, one column
+  // per thread -> J buffer.  Q = G D^-1 X with X[piv_a][:] = U[a][:] has orthonormal columns and
+  // Q^T g_i = f_i, so Aacc starts as D^-1 X (p x r).
+  for (int bcol = c.tid; bcol < r; bcol += c.nt) {
+    for (int a = bcol; a >= 0; --a) {
+      const int pa = (int)s.wused[a];
+      double acc = (a == bcol) ? 1.0 : 0.0;
+      for (int l = a + 1; l <= bcol; ++l) acc -= s.P[a * ld + (int)s.wused[l]] * s.J[l * ld + bcol];
+      s.J[a * ld + bcol] = acc / s.P[a * ld + pa];
+    }
   }
   c.sync();
+  for (int idx = c.tid; idx < r * r; idx += c.nt) {
+    const int a = idx / r, bcol = idx - a * r;
+    if (bcol >= a) {
+      const int pa = (int)s.wused[a];
+      s.Aacc[pa * ld + bcol] = s.dinv[pa] * s.J[a * ld + bcol];
+    }
+  }
+  // ---- P = F: scale column i of R back by ||g_i||
+  for (int idx = c.tid; idx < r * p; idx += c.nt) {
+    const int k = idx / p, i = idx - k * p;
+    s.P[k * ld + i] = (s.dinv[i] != 0.0) ? s.P[k * ld + i] / s.dinv[i] : 0.0;
+  }
+  c.sync();
+  int sw = 0;
   for (int i = c.tid; i < p; i += c.nt) {
     double acc = 0.0;
     for (int k = 0; k < r; ++k) { double v = s.P[k * ld + i]; acc += v * v; }
