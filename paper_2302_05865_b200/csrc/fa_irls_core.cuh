@@ -31,7 +31,16 @@
 #endif
 
 #ifndef FA_IRLS_HOST
-#define FA_RSQRT(x) rsqrt(x)
+// 1/sqrt(x) for normal positive x: hardware approximation (about 22 bits) and two Newton steps.
+__device__ __forceinline__ double fa_fast_rsqrt(double x) {
+  double y;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  const double hx = 0.5 * x;
+  y = y * fma(-hx * y, y, 1.5);
+  y = y * fma(-hx * y, y, 1.5);
+  return y;
+}
+#define FA_RSQRT(x) fa_fast_rsqrt(x)
 #else
 #define FA_RSQRT(x) (1.0 / sqrt(x))
 #endif
@@ -43,7 +52,7 @@ constexpr double kZeroNormRel = 1e-30; // K_ii <= this * max K_kk: zero gradient
 constexpr double kSamePairRel = 1e-12; // D_ij^2 <= this * (K_ii + K_jj): identical pair
 constexpr double kRankRel = 1e-12;     // eigenvalue <= this * largest: direction dropped
 constexpr double kJacobiTol = 1e-17;   // rotate when |a_pq| > tol * sqrt(|a_pp a_qq|)
-constexpr double kJacobiBig = 1e-8;    // sweep again while some rotated |a_pq| exceeded this (relative)
+constexpr double kJacobiBig = 1e-6;    // sweep again while some rotated |a_pq| exceeded this (relative)
 constexpr int kMaxSweeps = 40;
 constexpr int kMaxP = 64;
 
