@@ -88,8 +88,10 @@ def test_full_size_properties(fa, name):
     # principal angles between G^T A and G^T A2 from p-dim quantities: the cross Gram is A^T K A2
     orth = float(np.abs(Ah.T @ Kref @ Ah - np.eye(m)).max())
     assert orth < 1e-6
-    cross = np.linalg.svd(Ah.T @ Kref @ A2h, compute_uv=False)
-    ang = float(np.arccos(np.clip(cross.min(), -1.0, 1.0)))
+    # sine form: the part of G^T A2 outside span(G^T A) is G^T R with R = A2 - A (A^T K A2)
+    R = A2h - Ah @ (Ah.T @ Kref @ A2h)
+    sin2 = np.linalg.eigvalsh(R.T @ Kref @ R)
+    ang = float(np.arcsin(np.sqrt(np.clip(sin2.max(), 0.0, 1.0))))
     assert ang < TOL[w.dtype][1]
 
     # sampled outputs, one by one in fp64
