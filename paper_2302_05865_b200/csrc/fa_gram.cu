@@ -83,18 +83,33 @@ __device__ __forceinline__ void finish_gram(const Params& prm, int* smem_flag) {
   const int p = prm.p, ntri = p * (p + 1) / 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nb = gridDim.x;
-  for (int c = warp; c < ntri; c += nwarps) {
-    const double* src = prm.partials + (size_t)c * nb;
-    double sum = 0.0;
-    for (int b = lane; b < nb; b += 32) sum += __ldcg(src + b);
+  constexpr int E = 8;                           // entries a warp sums at once (independent loads in flight)
+  for (int c0 = warp * E; c0 < ntri; c0 += nwarps * E) {
+    double sum[E];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    for (int e = 0; e < E; ++e) sum[e] = 0.0;
+    for (int b = lane; b < nb; b += 32) {
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+        if (c0 + e < ntri) sum[e] += __ldcg(prm.partials + (size_t)(c0 + e) * nb + b);
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) sum[e] += __shfl_xor_sync(0xffffffffu, sum[e], off);
+    }
     if (lane == 0) {
-      int i = 0, r = c;
-      while (r >= p - i) { r -= p - i; ++i; }
-      const int j = i + r;
-      prm.K[i * p + j] = sum;
-      prm.K[j * p + i] = sum;
+#pragma unroll
+      for (int e = 0; e < E; ++e) {
+        const int c = c0 + e;
+        if (c < ntri) {
+          int i = 0, r = c;
+          while (r >= p - i) { r -= p - i; ++i; }
+          const int j = i + r;
+          prm.K[i * p + j] = sum[e];
+          prm.K[j * p + i] = sum[e];
+        }
+      }
     }
   }
   if (threadIdx.x == 0) *prm.counter = 0u;     // leave the counter ready for the next launch
