@@ -10,6 +10,7 @@
 // accumulators.  Block totals go to the workspace; the last block to finish adds them up in a
 // fixed order and writes K, so the result is bit-reproducible and no second launch is needed.
 #include "fa_common.cuh"
+#include "fa_gram_finish.cuh"
 #include "fa_kernels.h"
 
 namespace fa {
@@ -34,10 +35,6 @@ struct Params {
   double* K;           // out: p x p, written by the last block to finish
   int* status;
 };
-
-__host__ __device__ inline int canon_index(int i, int j, int p) {   // i <= j
-  return i * p - (i * (i - 1)) / 2 + (j - i);
-}
 
 // Butterfly reduce-scatter of NACCP values per lane across the warp: afterwards lane l holds the
 // warp sums of elements [l*NACCP/32, (l+1)*NACCP/32) in x[0 .. NACCP/32).  NACCP is a multiple of 32.
@@ -64,55 +61,6 @@ __device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP 
   for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
 #pragma unroll
   for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
-}
-
-// Called by every thread of a block after it has written its entries of `partials`.  The last
-// block to arrive (atomic counter) adds up all blocks' entries and writes the symmetric K.  Each
-// entry is summed by one warp: lane l takes blocks l, l+32, ... in order, then a fixed shuffle
-// tree -- the order does not depend on which block happens to be last, so K is bit-reproducible.
-__device__ __forceinline__ void finish_gram(const Params& prm, int* smem_flag) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    const unsigned int done = atomicAdd(prm.counter, 1u);
-    *smem_flag = (done == gridDim.x - 1) ? 1 : 0;
-  }
-  __syncthreads();
-  if (!*smem_flag) return;
-  __threadfence();
-  const int p = prm.p, ntri = p * (p + 1) / 2;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  const int nb = gridDim.x;
-  constexpr int E = 8;                           // entries a warp sums at once (independent loads in flight)
-  for (int c0 = warp * E; c0 < ntri; c0 += nwarps * E) {
-    double sum[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) sum[e] = 0.0;
-    for (int b = lane; b < nb; b += 32) {
-#pragma unroll
-      for (int e = 0; e < E; ++e)
-        if (c0 + e < ntri) sum[e] += __ldcg(prm.partials + (size_t)(c0 + e) * nb + b);
-    }
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) sum[e] += __shfl_xor_sync(0xffffffffu, sum[e], off);
-    }
-    if (lane == 0) {
-#pragma unroll
-      for (int e = 0; e < E; ++e) {
-        const int c = c0 + e;
-        if (c < ntri) {
-          int i = 0, r = c;
-          while (r >= p - i) { r -= p - i; ++i; }
-          const int j = i + r;
-          prm.K[i * p + j] = sum[e];
-          prm.K[j * p + i] = sum[e];
-        }
-      }
-    }
-  }
-  if (threadIdx.x == 0) *prm.counter = 0u;     // leave the counter ready for the next launch
 }
 
 struct Ring {
@@ -284,7 +232,7 @@ __global__ void __launch_bounds__((CW + 1) * 32, 1) gram_tri_kernel(Params prm) 
       prm.partials[(size_t)canon_index(i, j, prm.p) * gridDim.x + blockIdx.x] = sum;
     }
   }
-  finish_gram(prm, ring.abort);
+  finish_gram(prm.partials, prm.counter, prm.K, prm.p, ring.abort);
 }
 
 // ---- consumers, 16 < p <= 64: rows are cut into blocks of 16; a work item is the triangle of
@@ -441,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_blocks_kernel(Params prm) {
     }
     prm.partials[(size_t)canon_index(gi, gj, prm.p) * gridDim.x + blockIdx.x] = sum;
   }
-  finish_gram(prm, ring.abort);
+  finish_gram(prm.partials, prm.counter, prm.K, prm.p, ring.abort);
 }
 
 // ---- host side
@@ -506,13 +454,12 @@ static cudaError_t dispatch(const Shape& sh, int vec, const Params& prm, int gri
 
 }  // namespace gram
 
+// Upper bound on the blocks any Gram kernel launches for this shape (one per SM at most); it
+// sizes the per-block partial sums in the workspace.
 int gram_num_blocks(int p, long long n, int dtype) {
-  const gram::Shape sh = gram::pick_shape(p);
-  const int S = dtype == 0 ? 4 : 2;
-  const long long tile_cols = sh.row_bytes / S;
-  const long long tiles = (n + tile_cols - 1) / tile_cols;
+  (void)p; (void)dtype;
   const int sms = sm_count();
-  return (int)(tiles < sms ? tiles : sms);
+  return (int)(n < sms ? n : sms);
 }
 
 size_t gram_partials_bytes(int p, long long n, int dtype) {
@@ -521,6 +468,7 @@ size_t gram_partials_bytes(int p, long long n, int dtype) {
 
 cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
                         double* K, int* status, cudaStream_t st) {
+  if (gram_tc_eligible(G, dtype, p, n)) return launch_gram_tc(G, p, n, partials, counter, K, status, st);
   const gram::Shape sh = gram::pick_shape(p);
   const int S = dtype == 0 ? 4 : 2;
   gram::Params prm{};
@@ -534,7 +482,8 @@ cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* pa
   prm.counter = counter;
   prm.K = K;
   prm.status = status;
-  const int grid = gram_num_blocks(p, n, dtype);
+  const int sms = sm_count();
+  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
   cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
   if (e != cudaSuccess) return e;
   // two elements per shared load when every row starts on an even element

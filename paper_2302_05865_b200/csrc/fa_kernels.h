@@ -14,6 +14,11 @@ size_t gram_partials_bytes(int p, long long n, int dtype);
 cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
                         double* K, int* status, cudaStream_t st);
 
+// Tensor-core Gram pass (bf16, 16 < p <= 64, 16-byte aligned rows); same scratch and output.
+bool gram_tc_eligible(const void* G, int dtype, int p, long long n);
+cudaError_t launch_gram_tc(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
+                           int* status, cudaStream_t st);
+
 // Persistent single-block IRLS on K (p x p).
 struct IrlsArgs {
   const double* K;

