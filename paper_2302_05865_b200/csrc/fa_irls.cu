@@ -30,9 +30,15 @@ static cudaError_t launch_nt(const IrlsArgs& a, cudaStream_t st) {
 // One thread per Jacobi work item where the block size allows it: (p/2)^2 2x2 blocks plus
 // p * p/2 eigenvector row pairs.
 cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
+#ifndef FA_IRLS_NT32
+#define FA_IRLS_NT32 512
+#endif
+#ifndef FA_IRLS_NT64
+#define FA_IRLS_NT64 512
+#endif
   if (a.p <= 16) return launch_nt<192>(a, st);
-  if (a.p <= 32) return launch_nt<768>(a, st);
-  return launch_nt<1024>(a, st);
+  if (a.p <= 32) return launch_nt<FA_IRLS_NT32>(a, st);
+  return launch_nt<FA_IRLS_NT64>(a, st);
 }
 
 }  // namespace fa

@@ -181,6 +181,68 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
 #ifndef FA_IRLS_HOST
+      if (np > 8) {
+        // Larger problems: the np rotations are computed once, by the first np threads, and published
+        // in shared memory (one extra barrier); redundant fp64 work would otherwise fill the pipe.
+        // Items are then taken three at a time, all loads first, so their latencies overlap.
+        if (c.tid < np) {
+          int a, b;
+          double cs, sn;
+          pair_of(rd, c.tid, pp, a, b);
+          if (rotation(T, ld, a, b, dim, cs, sn)) *big = 1;
+          s.ra[c.tid] = a; s.rb[c.tid] = b; s.rc[c.tid] = cs; s.rs[c.tid] = sn;
+        }
+        c.sync();
+        const int total = nblk + nrow;
+#ifndef FA_IRLS_BATCH
+#define FA_IRLS_BATCH 2
+#endif
+        constexpr int U = FA_IRLS_BATCH;
+        for (int base = c.tid; base < total; base += U * c.nt) {
+          int kind[U], ia[U], ib[U], ic[U], id[U];
+          double rk_c[U], rk_s[U], rl_c[U], rl_s[U], x0[U], x1[U], x2[U], x3[U];
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            const int idx = base + u * c.nt;
+            kind[u] = 0;
+            if (idx < nblk) {
+              const int k = idx >> sh, l = idx & mask;
+              if (l < np) {
+                kind[u] = 1;
+                ia[u] = s.ra[k]; ib[u] = s.rb[k]; ic[u] = s.ra[l]; id[u] = s.rb[l];
+                rk_c[u] = s.rc[k]; rk_s[u] = s.rs[k]; rl_c[u] = s.rc[l]; rl_s[u] = s.rs[l];
+                x0[u] = T[ia[u] * ld + ic[u]]; x1[u] = T[ia[u] * ld + id[u]];
+                x2[u] = T[ib[u] * ld + ic[u]]; x3[u] = T[ib[u] * ld + id[u]];
+                if (k == l && rk_s[u] != 0.0) kind[u] = 3;   // diagonal block: the rotated entry is exactly zero
+              }
+            } else if (idx < total) {
+              const int q = idx - nblk;
+              const int x = q >> sh, k = q & mask;
+              if (k < np && s.rs[k] != 0.0) {
+                kind[u] = 2;
+                ia[u] = x * ld + s.ra[k]; ib[u] = x * ld + s.rb[k];
+                rk_c[u] = s.rc[k]; rk_s[u] = s.rs[k];
+                x0[u] = J[ia[u]]; x1[u] = J[ib[u]];
+              }
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            if (kind[u] == 1 || kind[u] == 3) {
+              const double yac = rk_c[u] * x0[u] - rk_s[u] * x2[u], yad = rk_c[u] * x1[u] - rk_s[u] * x3[u];
+              const double ybc = rk_s[u] * x0[u] + rk_c[u] * x2[u], ybd = rk_s[u] * x1[u] + rk_c[u] * x3[u];
+              double zac = rl_c[u] * yac - rl_s[u] * yad, zad = rl_s[u] * yac + rl_c[u] * yad;
+              double zbc = rl_c[u] * ybc - rl_s[u] * ybd, zbd = rl_s[u] * ybc + rl_c[u] * ybd;
+              if (kind[u] == 3) { zad = 0.0; zbc = 0.0; }
+              Tn[ia[u] * ld + ic[u]] = zac; Tn[ia[u] * ld + id[u]] = zad;
+              Tn[ib[u] * ld + ic[u]] = zbc; Tn[ib[u] * ld + id[u]] = zbd;
+            } else if (kind[u] == 2) {
+              J[ia[u]] = rk_c[u] * x0[u] - rk_s[u] * x1[u];
+              J[ib[u]] = rk_s[u] * x0[u] + rk_c[u] * x1[u];
+            }
+          }
+        }
+      } else {
       // Items are strided by the block size, a multiple of the (power-of-two) pair count, so a
       // thread always meets the same column pair l: it computes that one rotation per round and
       // fetches the row pair's rotation from the lane that owns it (lane k of its own warp).
@@ -217,6 +279,7 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
           J[x * ld + bl] = sl * va + cl * vb;
         }
       }
+      }   // np <= 8
 #else
       for (int idx = c.tid; idx < nblk + nrow; idx += c.nt) {
         if (idx < nblk) {
