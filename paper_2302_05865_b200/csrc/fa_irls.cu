@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   fa_irls::Smem s;
   fa_irls::carve(s, irls_smem, a.p, ctx.nt);
   fa_irls::Outputs o{a.A, a.c, a.w, a.obj, a.status};
-  const int st = fa_irls::run(ctx, s, K, a.p, a.m, a.lambda, a.iters, a.start_from_A != 0, o);
+  const int st = fa_irls::run<(NT > 192)>(ctx, s, K, a.p, a.m, a.lambda, a.iters, a.start_from_A != 0, o);
   if (st && a.status && ctx.tid == 0) atomicOr(a.status, st);
 }
 

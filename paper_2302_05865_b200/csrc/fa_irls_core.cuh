@@ -161,6 +161,7 @@ FA_FN bool rotation(const double* T, int ld, int a, int b, int dim, double& cs, 
 // its diagonal: that sweep's rotations leave entries of the order of its square (quadratic
 // convergence of the cyclic method), i.e. below rounding level.
 // On return *Tio points at the buffer that holds the diagonalised matrix.  Returns the sweeps made.
+template <bool LARGE>
 FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double* J, int dim, int jrows) {
   const int ld = s.ld;
   const int pp = (dim + 1) & ~1;
@@ -181,7 +182,7 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
 #ifndef FA_IRLS_HOST
-      if (np > 8) {
+      if (LARGE && np > 8) {
         // Larger problems: the np rotations are computed once, by the first np threads, and published
         // in shared memory (one extra barrier); redundant fp64 work would otherwise fill the pipe.
         // Items are then taken three at a time, all loads first, so their latencies overlap.
@@ -423,6 +424,7 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
 // K: p x p inner products (global or shared memory).  start_from_A: take the subspace in o.A as
 // the current one for the first reweighting (single-step interface); otherwise round one is
 // uniform.  Returns the status bits (same value in every thread).
+template <bool LARGE>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, int iters,
               bool start_from_A, const Outputs& o) {
   const int ld = s.ld;
@@ -601,7 +603,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       if (a >= r || b >= r) s.T[a * ld + b] = 0.0;
     }
     c.sync();
-    sw = jacobi(c, s, &s.T, &s.tmp, s.J, r, r);
+    sw = jacobi<LARGE>(c, s, &s.T, &s.tmp, s.J, r, r);
     if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
     m_eff = sort_eigs(c, s, s.T, r, m);
 
