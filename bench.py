@@ -42,8 +42,9 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs (read-only)."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """nvidia-smi clock / throttle-reason samples (read-only queries), time-stamped so that only the
+    samples taken while the timed region ran are used."""
+    QUERY = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -56,12 +57,15 @@ class ClockSampler:
         try:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and the set of active slow-down reasons over [t_begin, t_end] (time.time()
+        values); falls back to the samples closest to the window when none fell inside it."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -72,23 +76,34 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        rows = []
         for line in self.file.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 9:
+            if len(parts) < 10:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[2]), float(parts[3]), parts[6:10]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
-                                 parts[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.file.close()
         os.unlink(self.file.name)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        if not rows:
+            return out
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        if not inside and t_begin is not None:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:2]
+            out["note"] = "no sample fell inside the timed region; nearest samples used"
+        if not inside:
+            inside = rows
+        reasons = set()
+        for r in inside:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        out.update(sm_mhz=statistics.median(r[1] for r in inside), sm_max_mhz=max(r[2] for r in inside),
+                   reasons=sorted(reasons), samples=len(inside))
         return out
 
 
@@ -154,7 +169,7 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(si.WORKLOADS))
@@ -206,19 +221,22 @@ def main():
 
     for i in range(args.warmup):
         step(i)
-    barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+    for i in range(args.warmup):          # second warm-up batch while the clock sampler spins up
+        step(i)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_begin = time.time()
     ev0.record(stream)
     for i in range(args.steps):
         step(i)
     ev1.record(stream)
     barrier()
+    t_end = time.time()
     elapsed_ms = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     if int(status.item()) != 0:
         raise SystemExit(f"device status {int(status.item())} after the timed region")
     if world > 1:
@@ -249,6 +267,9 @@ def main():
     t_irls = time_call(lambda i: fa.fa_irls(K, w.m, w.lam, w.iters, c_out=cvec, stream=stream), reps)
 
     peak, peak_src = measured_peaks()
+    # DRAM bytes per Gram launch from the ncu capture summarised in profiles/gram_tri_f32_p15_cfg2.md
+    # (246.4 MB at n = 4,000,000, scaled by n); only valid for that kernel and workload
+    traffic = int(246.4e6 * w.n / 4_000_000) if (w.p == 15 and w.dtype == "f32") else None
     gram_bytes = w.p * w.n * w.itemsize
     comb_bytes = w.p * w.n * w.itemsize + 4 * w.n
     gram_gbs = gram_bytes / (t_gram * 1e-3) / 1e9
@@ -301,7 +322,7 @@ def main():
                    "storage": w.dtype, "l2": f"inputs larger than L2; {nbuf} device copies of G rotated between steps",
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
         "roofline": {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
-                     "unit": "GB/s", "frac": gram_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "unit": "GB/s", "frac": gram_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_launch": int(gram_bytes), "ms_per_launch": t_gram},
         "kernels": {"gram_ms": t_gram, "irls_ms": t_irls, "combine_ms": t_comb,
                     "combine_gbs": comb_gbs, "combine_frac": comb_gbs / peak},
