@@ -135,14 +135,19 @@ def term_values(G, Y, lam, norms=None, zero=None, D2=None, active=None):
     return u, U
 
 
-def objective(G, Y, lam) -> float:
-    """A(Y) of Eq. (5) with regulariser (2); the pair sum runs over ordered pairs."""
+def objective(G, Y, lam, a=2.0) -> float:
+    """A(Y) of Eq. (5) with regulariser (2); the pair sum runs over ordered pairs.
+
+    a is the constant of the Taylor surrogate of Eq. (4): each term is (1 - v)^(1/a); a = 2 (the
+    paper's choice, Section 2.3) gives the square roots of Eq. (5).  The constant factor a and
+    the offset -a of Eq. (4) do not move the minimiser and are left out.
+    """
     G = np.asarray(G, dtype=np.float64)
     p = G.shape[0]
     u, U = term_values(G, Y, lam)
-    val = float(np.sum(np.sqrt(np.maximum(u, 0.0))))
+    val = float(np.sum(np.maximum(u, 0.0) ** (1.0 / a)))
     if lam > 0 and p > 1:
-        val += lam / (p - 1) * float(np.sum(np.sqrt(np.maximum(U, 0.0))))
+        val += lam / (p - 1) * float(np.sum(np.maximum(U, 0.0) ** (1.0 / a)))
     return val
 
 
@@ -204,10 +209,13 @@ def weighted_pca_svd(G, w, W, m):
 
 # -- the iteration -------------------------------------------------------------
 
-def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False):
+def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a=2.0):
     """Run `iters` IRLS rounds and return the aggregate.
 
     G      : (p, n) array, rows are worker gradients (converted to float64)
+    a      : surrogate constant of Eq. (4), a > 1; terms are (1 - v)^(1/a) and the reweighting
+             of a term with value u is 1 / (normaliser * max(u^(1 - 1/a), eps))  (a = 2: the paper's
+             square roots)
     returns: dict with d (n,), Y (n, k<=m), u (p,), w (p,) last data weights,
              objective (list, one per round), evals (last round, descending),
              and with history=True the list of Y per round.
@@ -216,8 +224,8 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False):
     p, n = G.shape
     if not (1 <= m <= p):
         raise ValueError("need 1 <= m <= p")
-    if iters < 1 or lam < 0:
-        raise ValueError("need iters >= 1 and lam >= 0")
+    if iters < 1 or lam < 0 or not (a > 1.0):
+        raise ValueError("need iters >= 1, lam >= 0 and a > 1")
     norms, zero = _classify(G)
     D2, active = _pairs(G, norms, lam)
     coef = lam / (p - 1) if (lam > 0 and p > 1) else 0.0
@@ -237,21 +245,27 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False):
             w[~zero] = 1.0
             W[active] = coef
         else:
-            r = np.sqrt(np.maximum(u, 0.0))
+            r = np.maximum(u, 0.0) ** (1.0 - 1.0 / a)
             w[~zero] = 1.0 / (norms[~zero] * np.maximum(r[~zero], eps))
             if coef > 0:
-                R = np.sqrt(np.maximum(U, 0.0))
+                R = np.maximum(U, 0.0) ** (1.0 - 1.0 / a)
                 W[active] = coef / (D2[active] * np.maximum(R[active], eps))
         Y, evals = pca(G, w, W, m)
         u, U = term_values(G, Y, lam, norms, zero, D2, active)
-        obj = float(np.sum(np.sqrt(np.maximum(u, 0.0))))
+        obj = float(np.sum(np.maximum(u, 0.0) ** (1.0 / a)))
         if coef > 0:
-            obj += coef * float(np.sum(np.sqrt(np.maximum(U, 0.0))))
+            obj += coef * float(np.sum(np.maximum(U, 0.0) ** (1.0 / a)))
         objs.append(obj)
         if history:
             Ys.append(Y)
     d = Y @ (Y.T @ G.sum(axis=0)) / p
     return dict(d=d, Y=Y, u=u, w=w, objective=objs, evals=evals, Ys=Ys)
+
+
+def reconstruction(G, Y):
+    """Y Y^T g_i for every worker, as rows (the reconstruction Y Y^T G of Section 2.1, transposed)."""
+    G = np.asarray(G, dtype=np.float64)
+    return (G @ Y) @ Y.T
 
 
 # -- comparison helpers ----------------------------------------------------------

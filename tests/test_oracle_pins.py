@@ -374,3 +374,63 @@ def test_inner_products_and_pair_distances():
         for j in range(5):
             assert abs(K[i, j] - sum(G[i, k] * G[j, k] for k in range(17))) < 1e-10
             assert abs(D2[i, j] - (K[i, i] + K[j, j] - 2 * K[i, j])) < 1e-9
+
+
+# 14 -- other surrogate constants a (Eq. (4)): a = 2 is the default path; for a != 2 the iteration
+# still descends on sum (1 - v)^(1/a) and its limit is a local minimiser of that objective
+def eq4_objective(G, Y, lam, a):
+    p = G.shape[0]
+    val = 0.0
+    for i in range(p):
+        x = G[i]
+        if x @ x > 0:
+            val += max(1.0 - np.sum((Y.T @ x) ** 2) / (x @ x), 0.0) ** (1.0 / a)
+    if lam > 0:
+        for i in range(p):
+            for j in range(p):
+                if i != j:
+                    x = G[i] - G[j]
+                    if x @ x > 0:
+                        val += lam / (p - 1) * max(1.0 - np.sum((Y.T @ x) ** 2) / (x @ x), 0.0) ** (1.0 / a)
+    return val
+
+
+def test_surrogate_constant_two_is_the_default():
+    G = noisy_mean(8, 30, 90, outliers=2)
+    a2 = fo.fa_aggregate(G, 3, 0.1, iters=6, a=2.0)
+    d = fo.fa_aggregate(G, 3, 0.1, iters=6)
+    assert np.array_equal(a2["d"], d["d"]) and a2["objective"] == d["objective"]
+
+
+@pytest.mark.parametrize("a,lam", [(1.5, 0.0), (3.0, 0.3), (4.0, 0.0)])
+def test_other_surrogate_constants_descend_and_reach_a_local_minimum(a, lam):
+    n, p, m = 12, 10, 3
+    G = noisy_mean(p, n, 91, sigma=0.6, outliers=2, scale_spread=True)
+    out = fo.fa_aggregate(G, m, lam, iters=400, a=a)
+    obj = np.array(out["objective"])
+    assert np.all(np.diff(obj) <= 1e-10)
+    # the typed-out form 1 - v cancels: a captured worker's term carries rounding noise 1e-16^(1/a)
+    assert abs(obj[-1] - eq4_objective(G, out["Y"], lam, a)) < 10 * p * (1e-15 ** (1.0 / a))
+    Y = out["Y"]
+    base = eq4_objective(G, Y, lam, a)
+    r = rng(92)
+    worst = 0.0
+    for _ in range(40):
+        D = r.standard_normal((n, m))
+        D -= Y @ (Y.T @ D)
+        D /= np.linalg.norm(D)
+        for t in (1e-2, 1e-3):
+            Q, _ = np.linalg.qr(Y + t * D)
+            worst = max(worst, (base - eq4_objective(G, Q, lam, a)) / t)
+    assert worst < 1e-3
+
+
+# 15 -- reconstruction Y Y^T G (Section 2.1) is a projection of every gradient onto span(Y)
+def test_reconstruction_is_the_orthogonal_projection():
+    G = noisy_mean(6, 25, 93, outliers=1)
+    out = fo.fa_aggregate(G, 3, 0.0, iters=4)
+    R = fo.reconstruction(G, out["Y"])
+    P = out["Y"] @ out["Y"].T
+    assert np.allclose(R, G @ P, atol=1e-12)
+    assert np.allclose(R.mean(axis=0), out["d"], atol=1e-12)          # its column average is the update
+    assert np.allclose((G - R) @ out["Y"], 0.0, atol=1e-10)           # residuals are orthogonal to Y
