@@ -92,6 +92,17 @@ int fa_irls(const double* K, int p, int m, double lambda, int iters,
             double* A_out, float* c_out, double* w_out, double* obj_out,
             int* status, void* stream);
 
+/* fa_irls with two more knobs (next steps the paper names beyond its own settings):
+ *   a     : constant of the Taylor surrogate of Eq. (4), a > 1.  Each term of the objective is
+ *           (1 - v)^(1/a) and the reweighting of a term with value u is 1/(normaliser * max(u^(1-1/a), 1e-6));
+ *           a = 2 is the paper's choice (Section 2.3) and what fa_irls uses.
+ *   S_out : out p x p fp64 row-major or NULL, the "flag selection" matrix of the appendix's optimality
+ *           conditions: Y Y^T G = G S in the paper's layout, i.e. the reconstruction of worker j is
+ *           sum_i S[i][j] g_i, and c = (1/p) S 1. */
+int fa_irls_ex(const double* K, int p, int m, double lambda, double a, int iters,
+               double* A_out, float* c_out, double* S_out, double* w_out, double* obj_out,
+               int* status, void* stream);
+
 /* out[j] = sum_i c[i] * G[i][j]  (Algorithm 1 direction step in its right-multiplied form).
  * One streaming read of G, one write of n floats.  c: p floats on the device. */
 int fa_combine(const void* G, int dtype, int p, long long n, const float* c,
@@ -104,6 +115,11 @@ int fa_combine(const void* G, int dtype, int p, long long n, const float* c,
 int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lambda,
                  int iters, float* out, double* A_out, void* ws, size_t ws_bytes,
                  int* status, void* stream);
+
+/* fa_aggregate with the surrogate constant a and the selection matrix S_out of fa_irls_ex. */
+int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double lambda, double a,
+                    int iters, float* out, double* A_out, double* S_out, void* ws, size_t ws_bytes,
+                    int* status, void* stream);
 
 /* The same step for gradients that sit in HOST memory (Algorithm 1: the server receives the
  * gradients, aggregates, sends d back).  Enqueues on `stream`: copy G_host -> G_dev, the three

@@ -32,12 +32,14 @@ _lib.fa_workspace_bytes.argtypes = [_i, _ll, _i, _i, ctypes.POINTER(_sz)]
 _lib.fa_gram.argtypes = [_vp, _i, _i, _ll, _vp, _vp, _sz, _vp]
 _lib.fa_irls_step.argtypes = [_vp, _i, _i, _d, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_irls.argtypes = [_vp, _i, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.fa_irls_ex.argtypes = [_vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.fa_aggregate_ex.argtypes = [_vp, _i, _i, _ll, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_combine.argtypes = [_vp, _i, _i, _ll, _vp, _vp, _vp]
 _lib.fa_aggregate.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_aggregate_host.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_gram_static.argtypes = [_vp, _i, _i, _ll, _vp, _vp]
 _lib.fa_gram_static.restype = _i
-for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_combine", "fa_aggregate",
+for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_irls_ex", "fa_aggregate_ex", "fa_combine", "fa_aggregate",
               "fa_aggregate_host"):
     getattr(_lib, _name).restype = _i
 
@@ -128,6 +130,34 @@ def fa_irls(K, m, lam, iters, A_out=None, c_out=None, w_out=None, obj_out=None, 
                         _dev(c_out, torch.float32, p, "c_out"), _ptr(w_out), _ptr(obj_out), _ptr(status),
                         _stream(stream)), "fa_irls")
     return c_out
+
+
+def fa_irls_ex(K, m, lam, a, iters, A_out=None, c_out=None, S_out=None, w_out=None, obj_out=None, status=None,
+               stream=None):
+    """fa_irls with the surrogate constant a (a = 2: the paper's) and the p x p selection matrix S_out."""
+    p = int(K.shape[0])
+    c_out = torch.empty(p, dtype=torch.float32, device=K.device) if c_out is None else c_out
+    if S_out is not None:
+        _dev(S_out, torch.float64, p * p, "S_out")
+    _check(_lib.fa_irls_ex(_dev(K, torch.float64, p * p, "K"), p, m, float(lam), float(a), iters, _ptr(A_out),
+                           _dev(c_out, torch.float32, p, "c_out"), _ptr(S_out), _ptr(w_out), _ptr(obj_out),
+                           _ptr(status), _stream(stream)), "fa_irls_ex")
+    return c_out
+
+
+def fa_aggregate_ex(G, m, lam, a, iters, out=None, A_out=None, S_out=None, ws=None, status=None, stream=None):
+    """fa_aggregate with the surrogate constant a and the selection matrix S_out."""
+    code, p, n = _gradients(G)
+    out = torch.empty(n, dtype=torch.float32, device=G.device) if out is None else out
+    ws = new_workspace(G, m) if ws is None else ws
+    if A_out is not None:
+        _dev(A_out, torch.float64, p * m, "A_out")
+    if S_out is not None:
+        _dev(S_out, torch.float64, p * p, "S_out")
+    _check(_lib.fa_aggregate_ex(G.data_ptr(), code, p, n, m, float(lam), float(a), iters,
+                                _dev(out, torch.float32, n, "out"), _ptr(A_out), _ptr(S_out), ws.data_ptr(),
+                                ws.numel() * ws.element_size(), _ptr(status), _stream(stream)), "fa_aggregate_ex")
+    return out
 
 
 def fa_combine(G, c, out=None, stream=None):

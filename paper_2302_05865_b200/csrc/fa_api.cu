@@ -96,22 +96,29 @@ int fa_irls_step(const double* K, int p, int m, double lambda, int first, double
       (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
   fa::IrlsArgs a{};
-  a.K = K; a.p = p; a.m = m; a.iters = 1; a.lambda = lambda; a.start_from_A = first ? 0 : 1;
+  a.K = K; a.p = p; a.m = m; a.iters = 1; a.lambda = lambda; a.a = 2.0; a.start_from_A = first ? 0 : 1;
   a.A = A; a.w = w; a.obj = objective; a.status = status;
   return fa::launch_irls(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
 
-int fa_irls(const double* K, int p, int m, double lambda, int iters, double* A_out, float* c_out, double* w_out,
-            double* obj_out, int* status, void* stream) {
-  if (!K || !c_out || p < 1 || p > FA_MAX_P || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda))
+int fa_irls_ex(const double* K, int p, int m, double lambda, double a, int iters, double* A_out, float* c_out,
+               double* S_out, double* w_out, double* obj_out, int* status, void* stream) {
+  if (!K || !c_out || p < 1 || p > FA_MAX_P || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda) ||
+      !(a > 1.0) || isinf(a))
     return FA_ERR_ARG;
   if (!fa::aligned(K, 8) || (A_out && !fa::aligned(A_out, 8)) || !fa::aligned(c_out, 4) ||
-      (w_out && !fa::aligned(w_out, 8)) || (obj_out && !fa::aligned(obj_out, 8)) || (status && !fa::aligned(status, 4)))
+      (S_out && !fa::aligned(S_out, 8)) || (w_out && !fa::aligned(w_out, 8)) || (obj_out && !fa::aligned(obj_out, 8)) ||
+      (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
-  fa::IrlsArgs a{};
-  a.K = K; a.p = p; a.m = m; a.iters = iters; a.lambda = lambda; a.start_from_A = 0;
-  a.A = A_out; a.c = c_out; a.w = w_out; a.obj = obj_out; a.status = status;
-  return fa::launch_irls(a, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+  fa::IrlsArgs args{};
+  args.K = K; args.p = p; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a; args.start_from_A = 0;
+  args.A = A_out; args.c = c_out; args.S = S_out; args.w = w_out; args.obj = obj_out; args.status = status;
+  return fa::launch_irls(args, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+int fa_irls(const double* K, int p, int m, double lambda, int iters, double* A_out, float* c_out, double* w_out,
+            double* obj_out, int* status, void* stream) {
+  return fa_irls_ex(K, p, m, lambda, 2.0, iters, A_out, c_out, nullptr, w_out, obj_out, status, stream);
 }
 
 int fa_combine(const void* G, int dtype, int p, long long n, const float* c, float* out, void* stream) {
@@ -121,26 +128,31 @@ int fa_combine(const void* G, int dtype, int p, long long n, const float* c, flo
                                                                                                        : FA_ERR_CUDA;
 }
 
-int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lambda, int iters, float* out,
-                 double* A_out, void* ws, size_t ws_bytes, int* status, void* stream) {
+int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double lambda, double a, int iters,
+                    float* out, double* A_out, double* S_out, void* ws, size_t ws_bytes, int* status, void* stream) {
   if (!G || !out || !ws || !fa::shape_ok(p, n, dtype) || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) ||
-      isinf(lambda))
+      isinf(lambda) || !(a > 1.0) || isinf(a))
     return FA_ERR_ARG;
   if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(out, 4) || (A_out && !fa::aligned(A_out, 8)) ||
-      !fa::aligned(ws, 16) || (status && !fa::aligned(status, 4)))
+      (S_out && !fa::aligned(S_out, 8)) || !fa::aligned(ws, 16) || (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
   fa::Workspace w = fa::carve_ws(ws, p, n, dtype);
   if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
   if (fa::launch_gram(G, dtype, p, n, w.partials, w.counter, w.Kbuf, status, st) != cudaSuccess) return FA_ERR_CUDA;
-  fa::IrlsArgs a{};
-  a.K = w.Kbuf;
-  a.p = p; a.m = m; a.iters = iters; a.lambda = lambda; a.start_from_A = 0;
-  a.A = A_out; a.c = w.c; a.status = status;
-  if (fa::launch_irls(a, st) != cudaSuccess) return FA_ERR_CUDA;
+  fa::IrlsArgs args{};
+  args.K = w.Kbuf;
+  args.p = p; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a; args.start_from_A = 0;
+  args.A = A_out; args.c = w.c; args.S = S_out; args.status = status;
+  if (fa::launch_irls(args, st) != cudaSuccess) return FA_ERR_CUDA;
   if (fa::launch_combine(G, dtype, p, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
   return FA_OK;
+}
+
+int fa_aggregate(const void* G, int dtype, int p, long long n, int m, double lambda, int iters, float* out,
+                 double* A_out, void* ws, size_t ws_bytes, int* status, void* stream) {
+  return fa_aggregate_ex(G, dtype, p, n, m, lambda, 2.0, iters, out, A_out, nullptr, ws, ws_bytes, status, stream);
 }
 
 int fa_aggregate_host(const void* G_host, int dtype, int p, long long n, int m, double lambda, int iters,

@@ -353,11 +353,20 @@ FA_FN int sort_eigs(const Ctx& c, const Smem& s, const double* T, int dim, int l
   return keep;
 }
 
+// One term of the objective with value u (the quantity under the root in Eq. (5)): its
+// contribution u^(1/a) and the factor max(u^(1 - 1/a), eps) of its reweighting (Eq. (4) with
+// constant a; a = 2 gives the square roots of Eq. (5) and takes the sqrt fast path).
+FA_FN void term_of(double u, double a, double& contrib, double& denom) {
+  if (a == 2.0) { contrib = sqrt(u); denom = fmax(contrib, kEps); }
+  else if (u <= 0.0) { contrib = 0.0; denom = kEps; }
+  else { contrib = pow(u, 1.0 / a); denom = fmax(pow(u, 1.0 - 1.0 / a), kEps); }
+}
+
 // From residual coordinates Res (rows k0..r-1 are the part of f_i outside the subspace) and the
 // full coordinates P: u_i, next data weights w_i, the matrix M of the next weighted PCA and the
 // value of Eq. (5).  `uniform` builds the round-one weights instead (u is not needed then).
 FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
-                                   double coef, bool uniform) {
+                                   double coef, bool uniform, double a) {
   const int ld = s.ld;
   double part = 0.0;
   for (int i = c.tid; i < p; i += c.nt) {
@@ -368,9 +377,10 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
         double acc = 0.0;
         for (int k = k0; k < r; ++k) { double v = Res[k * ld + i]; acc += v * v; }
         ui = acc / s.fn[i];
-        double root = sqrt(ui);
-        part += root;
-        wi = 1.0 / (s.fn[i] * fmax(root, kEps));
+        double contrib, denom;
+        term_of(ui, a, contrib, denom);
+        part += contrib;
+        wi = 1.0 / (s.fn[i] * denom);
       }
     }
     s.u[i] = ui;
@@ -389,9 +399,10 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
         if (uniform) wij = coef;
         else {
           for (int k = k0; k < r; ++k) { double v = Res[k * ld + i] - Res[k * ld + j]; res2 += v * v; }
-          double root = sqrt(res2 / d2);
-          part += coef * root;
-          wij = coef / (d2 * fmax(root, kEps));
+          double contrib, denom;
+          term_of(res2 / d2, a, contrib, denom);
+          part += coef * contrib;
+          wij = coef / (d2 * denom);
         }
       }
       s.M[i * ld + j] = -2.0 * wij;
@@ -412,6 +423,7 @@ struct Outputs {
   float* c;           // p or null
   double* w;          // p or null
   double* obj;        // iters (or 1) or null
+  double* S;          // p x p selection matrix or null
   int* status;        // or null
 };
 
@@ -419,13 +431,14 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
   for (int i = c.tid; i < p * m; i += c.nt) if (o.A) o.A[i] = 0.0;
   for (int i = c.tid; i < p; i += c.nt) { if (o.c) o.c[i] = 0.f; if (o.w) o.w[i] = 0.0; }
   for (int i = c.tid; i < iters; i += c.nt) if (o.obj) o.obj[i] = 0.0;
+  for (int i = c.tid; i < p * p; i += c.nt) if (o.S) o.S[i] = 0.0;
 }
 
 // K: p x p inner products (global or shared memory).  start_from_A: take the subspace in o.A as
 // the current one for the first reweighting (single-step interface); otherwise round one is
 // uniform.  Returns the status bits (same value in every thread).
 template <bool LARGE>
-FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, int iters,
+FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
               bool start_from_A, const Outputs& o) {
   const int ld = s.ld;
   const int pp = (p + 1) & ~1;
@@ -542,7 +555,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
 
   // ---- weights of the first round
   if (!start_from_A) {
-    (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true);
+    (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
   } else {
     // Z0 = F A (r x m) -> J buffer; C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
     for (int idx = c.tid; idx < r * m; idx += c.nt) {
@@ -566,7 +579,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       s.tmp[k * ld + i] = acc;
     }
     c.sync();
-    (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false);
+    (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a);
   }
 
   int m_eff = 0;
@@ -627,7 +640,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
 
     // ---- terms of Eq. (5) at the new subspace, and the next round's weights
-    double obj = weights_and_objective(c, s, s.P, m_eff, r, p, coef, false);
+    double obj = weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
   }
   if (m_eff < m) status |= ST_RANK_LT_M;
@@ -640,6 +653,14 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
   }
   if (o.w) for (int i = c.tid; i < p; i += c.nt) o.w[i] = s.wused[i];
+  if (o.S) {   // Y Y^T G = G S with S = A (A^T K): (A^T K) e_j are the leading coordinates of f_j
+    for (int idx = c.tid; idx < p * p; idx += c.nt) {
+      const int i = idx / p, j = idx - i * p;
+      double acc = 0.0;
+      for (int k = 0; k < m_eff; ++k) acc += s.Aacc[i * ld + k] * s.P[k * ld + j];
+      o.S[idx] = acc;
+    }
+  }
   if (o.c) {
     for (int k = c.tid; k < m_eff; k += c.nt) {        // s_k = sum_j P[k][j]  (Z^T F 1)
       double acc = 0.0;

@@ -24,11 +24,13 @@ struct IrlsArgs {
   const double* K;
   int p, m, iters;
   double lambda;
+  double a;          // surrogate constant of Eq. (4); 2 = the paper's square roots
   int start_from_A;
   double* A;
   float* c;
   double* w;
   double* obj;
+  double* S;         // p x p selection matrix or null
   int* status;
 };
 cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st);

@@ -130,6 +130,56 @@ def test_irls_rounds_match_oracle_from_exact_inner_products(fa, p, n, kind, m, l
         assert fo.principal_angles(ref["Y"], G.T @ A1.cpu().numpy()[:, :k]).max() < 1e-7
 
 
+EX_CASES = [
+    (1, 9, "noisy_mean", 1, 0.0, 1.5, 3), (3, 33, "dup_zero", 2, 0.2, 3.0, 5), (15, 2000, "noisy_mean", 8, 0.01, 1.5, 10),
+    (15, 2000, "noisy_mean", 8, 0.01, 4.0, 10), (16, 100, "gauss", 8, 0.1, 3.0, 6), (31, 3000, "noisy_mean", 12, 0.01, 2.5, 12),
+    (63, 200, "dup_zero", 16, 0.02, 1.25, 8), (64, 300, "noisy_mean", 20, 0.01, 2.0, 8),
+]
+
+
+@pytest.mark.parametrize("p,n,kind,m,lam,a,iters", EX_CASES)
+def test_irls_with_another_surrogate_constant_and_the_selection_matrix(fa, p, n, kind, m, lam, a, iters):
+    """Exponent 1/a of Eq. (4) with a != 2, and S with Y Y^T g_j = sum_i S[i][j] g_i."""
+    G = si.ladder_case(p, n, 9, kind).astype(np.float64)
+    ref = fo.fa_aggregate(G, m, lam, iters, a=a)
+    K = torch.from_numpy(fo.inner_products(G)).cuda()
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    S = torch.full((p, p), float("nan"), dtype=torch.float64, device="cuda")
+    w = torch.zeros(p, dtype=torch.float64, device="cuda")
+    obj = torch.zeros(iters, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = fa.fa_irls_ex(K, m, lam, a, iters, A_out=A, S_out=S, w_out=w, obj_out=obj, status=status)
+    torch.cuda.synchronize()
+    k = ref["Y"].shape[1]
+    assert int(status.item()) & ~fa.ST_RANK_LT_M == 0
+    Y = G.T @ A.cpu().numpy()[:, :k]
+    if k:
+        assert fo.principal_angles(ref["Y"], Y).max() < 1e-7
+    assert np.allclose(obj.cpu().numpy(), ref["objective"], rtol=1e-9, atol=1e-9)
+    assert np.allclose(w.cpu().numpy(), ref["w"], rtol=1e-6, atol=0)
+    assert fo.rel_l2(c.cpu().numpy().astype(np.float64) @ G, ref["d"]) < 1e-6
+    Sh = S.cpu().numpy()
+    R = fo.reconstruction(G, ref["Y"])
+    assert np.abs(Sh.T @ G - R).max() <= 1e-8 * max(1.0, np.abs(R).max())
+    assert np.allclose(Sh.sum(axis=1) / p, c.cpu().numpy(), rtol=1e-5, atol=1e-7)
+
+
+def test_aggregate_ex_equals_its_parts(fa):
+    G_np = si.ladder_case(15, 70_001, 4, "noisy_mean")
+    G = torch.from_numpy(G_np).cuda()
+    S = torch.zeros((15, 15), dtype=torch.float64, device="cuda")
+    out = fa.fa_aggregate_ex(G, 8, 0.01, 3.0, 7, S_out=S)
+    ref = fo.fa_aggregate(G_np.astype(np.float64), 8, 0.01, 7, a=3.0)
+    assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < 1e-4
+    R = fo.reconstruction(G_np.astype(np.float64), ref["Y"])
+    assert fo.rel_l2(S.cpu().numpy().T @ G_np.astype(np.float64), R) < 1e-4
+    assert torch.equal(fa.fa_aggregate_ex(G, 8, 0.01, 2.0, 7), fa.fa_aggregate(G, 8, 0.01, 7))
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate_ex(G, 8, 0.01, 1.0, 7)
+    with pytest.raises(fa.FaError):
+        fa.fa_irls_ex(torch.eye(3, dtype=torch.float64, device="cuda"), 2, 0.0, float("nan"), 3)
+
+
 def _aggregate_and_compare(fa, G_np, m, lam, iters, dtype_key, mis=0):
     from tests.gpu_util import to_device, redzones_intact, subspace_from_A
     p, n = G_np.shape
