@@ -121,6 +121,24 @@ int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double 
                     int iters, float* out, double* A_out, double* S_out, void* ws, size_t ws_bytes,
                     int* status, void* stream);
 
+/* Workers that hand in several gradients each (Section 2.1, "Advantages of Subspace based Aggregation";
+ * the extension paragraph of Section 2.2; the appendix restatement of Eq. (5) with
+ * tr(Y^T g_i g_i^T Y) / tr(g_i^T g_i)).  The `rows` gradients are the rows of G as before, the
+ * counts[i] >= 1 gradients of worker i being consecutive; counts is a HOST array of `workers`
+ * entries that add up to rows (read during the call, not kept), rows <= FA_MAX_P.
+ *   value of worker i : ratio of traces over its rows; one weight per worker on all of its rows;
+ *   regulariser       : pair terms between the workers' mean gradients, coefficient lambda/(workers-1);
+ *   aggregate         : (1/workers) Y Y^T (sum of the workers' mean gradients) = sum over rows of c * row.
+ * With every count equal to 1 this is fa_irls_ex / fa_aggregate_ex.  w_out has `workers` entries;
+ * A_out is rows x m, S_out rows x rows, c_out rows; m <= rows. */
+int fa_irls_multi(const double* K, int rows, const int* counts, int workers, int m, double lambda,
+                  double a, int iters, double* A_out, float* c_out, double* S_out, double* w_out,
+                  double* obj_out, int* status, void* stream);
+
+int fa_aggregate_multi(const void* G, int dtype, int rows, long long n, const int* counts, int workers,
+                       int m, double lambda, double a, int iters, float* out, double* A_out,
+                       double* w_out, void* ws, size_t ws_bytes, int* status, void* stream);
+
 /* The same step for gradients that sit in HOST memory (Algorithm 1: the server receives the
  * gradients, aggregates, sends d back).  Enqueues on `stream`: copy G_host -> G_dev, the three
  * kernels, copy out_dev -> out_host and, if both are given, status_dev -> status_host.

@@ -34,13 +34,15 @@ _lib.fa_irls_step.argtypes = [_vp, _i, _i, _d, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_irls.argtypes = [_vp, _i, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_irls_ex.argtypes = [_vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_aggregate_ex.argtypes = [_vp, _i, _i, _ll, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.fa_irls_multi.argtypes = [_vp, _i, _vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.fa_aggregate_multi.argtypes = [_vp, _i, _i, _ll, _vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_combine.argtypes = [_vp, _i, _i, _ll, _vp, _vp, _vp]
 _lib.fa_aggregate.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_aggregate_host.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_gram_static.argtypes = [_vp, _i, _i, _ll, _vp, _vp]
 _lib.fa_gram_static.restype = _i
-for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_irls_ex", "fa_aggregate_ex", "fa_combine", "fa_aggregate",
-              "fa_aggregate_host"):
+for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_irls_ex", "fa_aggregate_ex",
+              "fa_irls_multi", "fa_aggregate_multi", "fa_combine", "fa_aggregate", "fa_aggregate_host"):
     getattr(_lib, _name).restype = _i
 
 
@@ -157,6 +159,42 @@ def fa_aggregate_ex(G, m, lam, a, iters, out=None, A_out=None, S_out=None, ws=No
     _check(_lib.fa_aggregate_ex(G.data_ptr(), code, p, n, m, float(lam), float(a), iters,
                                 _dev(out, torch.float32, n, "out"), _ptr(A_out), _ptr(S_out), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), _ptr(status), _stream(stream)), "fa_aggregate_ex")
+    return out
+
+
+def _counts(counts):
+    return (ctypes.c_int * len(counts))(*[int(k) for k in counts])
+
+
+def fa_irls_multi(K, counts, m, lam, iters, a=2.0, A_out=None, c_out=None, S_out=None, w_out=None, obj_out=None,
+                  status=None, stream=None):
+    """IRLS rounds for workers that hold counts[i] consecutive rows of K each; returns c (one entry per row)."""
+    rows = int(K.shape[0])
+    arr = _counts(counts)
+    c_out = torch.empty(rows, dtype=torch.float32, device=K.device) if c_out is None else c_out
+    if w_out is not None:
+        _dev(w_out, torch.float64, len(counts), "w_out")
+    _check(_lib.fa_irls_multi(_dev(K, torch.float64, rows * rows, "K"), rows, arr, len(counts), m, float(lam), float(a),
+                              iters, _ptr(A_out), _dev(c_out, torch.float32, rows, "c_out"), _ptr(S_out), _ptr(w_out),
+                              _ptr(obj_out), _ptr(status), _stream(stream)), "fa_irls_multi")
+    return c_out
+
+
+def fa_aggregate_multi(G, counts, m, lam, iters, a=2.0, out=None, A_out=None, w_out=None, ws=None, status=None,
+                       stream=None):
+    """The whole step for workers with several gradients each (rows of one worker consecutive in G)."""
+    code, rows, n = _gradients(G)
+    arr = _counts(counts)
+    out = torch.empty(n, dtype=torch.float32, device=G.device) if out is None else out
+    ws = new_workspace(G, m) if ws is None else ws
+    if A_out is not None:
+        _dev(A_out, torch.float64, rows * m, "A_out")
+    if w_out is not None:
+        _dev(w_out, torch.float64, len(counts), "w_out")
+    _check(_lib.fa_aggregate_multi(G.data_ptr(), code, rows, n, arr, len(counts), m, float(lam), float(a), iters,
+                                   _dev(out, torch.float32, n, "out"), _ptr(A_out), _ptr(w_out), ws.data_ptr(),
+                                   ws.numel() * ws.element_size(), _ptr(status), _stream(stream)),
+           "fa_aggregate_multi")
     return out
 
 

@@ -55,6 +55,17 @@ bool shape_ok(int p, long long n, int dtype) {
 
 bool aligned(const void* ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
 
+// counts (host): `workers` positive entries that add up to `rows`
+bool counts_ok(const int* counts, int workers, int rows) {
+  if (!counts || workers < 1 || workers > rows) return false;
+  long long total = 0;
+  for (int i = 0; i < workers; ++i) {
+    if (counts[i] < 1 || counts[i] > rows) return false;
+    total += counts[i];
+  }
+  return total == rows;
+}
+
 }  // namespace
 }  // namespace fa
 
@@ -147,6 +158,45 @@ int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double 
   args.A = A_out; args.c = w.c; args.S = S_out; args.status = status;
   if (fa::launch_irls(args, st) != cudaSuccess) return FA_ERR_CUDA;
   if (fa::launch_combine(G, dtype, p, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
+  return FA_OK;
+}
+
+int fa_irls_multi(const double* K, int rows, const int* counts, int workers, int m, double lambda, double a, int iters,
+                  double* A_out, float* c_out, double* S_out, double* w_out, double* obj_out, int* status,
+                  void* stream) {
+  if (!K || !c_out || rows < 1 || rows > FA_MAX_P || !fa::counts_ok(counts, workers, rows) || m < 1 || m > rows ||
+      iters < 1 || !(lambda >= 0.0) || isinf(lambda) || !(a > 1.0) || isinf(a))
+    return FA_ERR_ARG;
+  if (!fa::aligned(K, 8) || (A_out && !fa::aligned(A_out, 8)) || !fa::aligned(c_out, 4) ||
+      (S_out && !fa::aligned(S_out, 8)) || (w_out && !fa::aligned(w_out, 8)) || (obj_out && !fa::aligned(obj_out, 8)) ||
+      (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::IrlsArgs args{};
+  args.K = K; args.p = rows; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a; args.start_from_A = 0;
+  args.A = A_out; args.c = c_out; args.S = S_out; args.w = w_out; args.obj = obj_out; args.status = status;
+  args.workers = workers;
+  for (int i = 0; i < workers; ++i) args.counts[i] = (unsigned char)counts[i];
+  return fa::launch_irls(args, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+int fa_aggregate_multi(const void* G, int dtype, int rows, long long n, const int* counts, int workers, int m,
+                       double lambda, double a, int iters, float* out, double* A_out, double* w_out, void* ws,
+                       size_t ws_bytes, int* status, void* stream) {
+  if (!G || !out || !ws || !fa::shape_ok(rows, n, dtype) || !fa::counts_ok(counts, workers, rows) || m < 1 ||
+      m > rows || iters < 1 || !(lambda >= 0.0) || isinf(lambda) || !(a > 1.0) || isinf(a))
+    return FA_ERR_ARG;
+  if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(out, 4) || (A_out && !fa::aligned(A_out, 8)) ||
+      (w_out && !fa::aligned(w_out, 8)) || !fa::aligned(ws, 16) || (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::Workspace w = fa::carve_ws(ws, rows, n, dtype);
+  if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_gram(G, dtype, rows, n, w.partials, w.counter, w.Kbuf, status, st) != cudaSuccess) return FA_ERR_CUDA;
+  int rc = fa_irls_multi(w.Kbuf, rows, counts, workers, m, lambda, a, iters, A_out, w.c, nullptr, w_out, nullptr, status,
+                         stream);
+  if (rc != FA_OK) return rc;
+  if (fa::launch_combine(G, dtype, rows, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
   return FA_OK;
 }
 

@@ -74,14 +74,19 @@ struct Smem {
   double *rc, *rs;                       // rotation cos / sin per pair
   int *ra, *rb, *ord;                    // rotation indices per pair, sort order
   int *flags;                            // [0],[3] rotated-this-sweep (by sweep parity), [1] scratch
+  // several gradients per worker (nw > 0): per-worker trace, value, weight, weight in use, 1/k_i;
+  // grp[row] = worker of a row, first[i] = first row of worker i
+  double *gtr, *gu, *gw, *gwused, *ginv;
+  int *grp, *first;
+  int nw;
   int ld;
 };
 
 FA_HD size_t smem_bytes(int p, int nt) {
   int pp = (p + 1) & ~1;
   int ld = pp + 1;
-  size_t doubles = (size_t)6 * pp * ld + (size_t)7 * pp + nt + 2 * (pp / 2 + 1);
-  size_t ints = (size_t)2 * (pp / 2 + 1) + pp + 8;
+  size_t doubles = (size_t)6 * pp * ld + (size_t)12 * pp + nt + 2 * (pp / 2 + 1);
+  size_t ints = (size_t)2 * (pp / 2 + 1) + 3 * pp + 8;
   return doubles * sizeof(double) + ints * sizeof(int) + 64;
 }
 
@@ -98,10 +103,13 @@ FA_FN void carve(Smem& s, void* base, int p, int nt) {
   s.tmp = d; d += (size_t)pp * ld;
   s.kd = d; d += pp; s.dinv = d; d += pp; s.fn = d; d += pp; s.u = d; d += pp;
   s.w = d; d += pp; s.wused = d; d += pp; s.ev = d; d += pp;
+  s.gtr = d; d += pp; s.gu = d; d += pp; s.gw = d; d += pp; s.gwused = d; d += pp; s.ginv = d; d += pp;
   s.red = d; d += nt;
   s.rc = d; d += pp / 2 + 1; s.rs = d; d += pp / 2 + 1;
   int* q = reinterpret_cast<int*>(d);
-  s.ra = q; q += pp / 2 + 1; s.rb = q; q += pp / 2 + 1; s.ord = q; q += pp; s.flags = q;
+  s.ra = q; q += pp / 2 + 1; s.rb = q; q += pp / 2 + 1; s.ord = q; q += pp; s.grp = q; q += pp;
+  s.first = q; q += pp; s.flags = q;
+  s.nw = 0;
 }
 
 // Deterministic block-wide sum; every thread gets the result.
@@ -418,6 +426,88 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
   return obj;
 }
 
+// The same for workers that hold several gradients each (rows of one worker are consecutive):
+// the value of worker i is 1 - tr(Y^T g_i g_i^T Y) / tr(g_i^T g_i) (appendix restatement of Eq. (5)),
+// one weight per worker multiplies all of its rows, and the pair terms of the regulariser are taken
+// between the workers' mean gradients.  `p` is the number of rows.  s.T and s.J are scratch here
+// (mean coordinates of every worker: all of them, and the residual part).
+FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
+                                           double coef, bool uniform, double a) {
+  const int ld = s.ld, nw = s.nw;
+  double* Fm = s.T;
+  double* Rm = s.J;
+  double part = 0.0;
+  double gmax = 0.0;
+  for (int i = 0; i < nw; ++i) gmax = fmax(gmax, s.gtr[i]);
+  for (int i = c.tid; i < nw; i += c.nt) {
+    double ui = 0.0, wi = 0.0;
+    if (s.gtr[i] > kZeroNormRel * gmax) {
+      if (uniform) wi = 1.0;
+      else {
+        const int r0 = s.first[i], r1 = (i + 1 < nw) ? s.first[i + 1] : p;
+        double acc = 0.0;
+        for (int row = r0; row < r1; ++row)
+          for (int k = k0; k < r; ++k) { double v = Res[k * ld + row]; acc += v * v; }
+        ui = acc / s.gtr[i];
+        double contrib, denom;
+        term_of(ui, a, contrib, denom);
+        part += contrib;
+        wi = 1.0 / (s.gtr[i] * denom);
+      }
+    }
+    s.gu[i] = ui;
+    s.gw[i] = wi;
+  }
+  if (coef > 0.0) {
+    for (int idx = c.tid; idx < r * nw; idx += c.nt) {
+      const int k = idx / nw, i = idx - k * nw;
+      const int r0 = s.first[i], r1 = (i + 1 < nw) ? s.first[i + 1] : p;
+      double fm = 0.0, rm = 0.0;
+      for (int row = r0; row < r1; ++row) { fm += s.P[k * ld + row]; rm += Res[k * ld + row]; }
+      Fm[k * ld + i] = fm * s.ginv[i];
+      Rm[k * ld + i] = (k >= k0) ? rm * s.ginv[i] : 0.0;
+    }
+  }
+  c.sync();
+  for (int row = c.tid; row < p; row += c.nt) { s.w[row] = s.gw[s.grp[row]]; s.u[row] = s.gu[s.grp[row]]; }
+  if (coef > 0.0) {
+    // rows of different workers i != j: M = -2 w_ij / (k_i k_j)  (ordered pairs: each pair twice)
+    for (int idx = c.tid; idx < p * p; idx += c.nt) {
+      const int ra = idx / p, rb = idx - ra * p;
+      const int i = s.grp[ra], j = s.grp[rb];
+      if (i == j) continue;
+      double d2 = 0.0, ni = 0.0, nj = 0.0, res2 = 0.0;
+      for (int k = 0; k < r; ++k) {
+        const double x = Fm[k * ld + i], y = Fm[k * ld + j];
+        d2 += (x - y) * (x - y); ni += x * x; nj += y * y;
+      }
+      double wij = 0.0;
+      if (d2 > kSamePairRel * (ni + nj)) {
+        if (uniform) wij = coef;
+        else {
+          for (int k = k0; k < r; ++k) { double v = Rm[k * ld + i] - Rm[k * ld + j]; res2 += v * v; }
+          double contrib, denom;
+          term_of(res2 / d2, a, contrib, denom);
+          if (ra == s.first[i] && rb == s.first[j]) part += coef * contrib;   // once per ordered pair
+          wij = coef / (d2 * denom);
+        }
+      }
+      s.M[ra * ld + rb] = -2.0 * wij * s.ginv[i] * s.ginv[j];
+    }
+    c.sync();
+    // rows of one worker: what makes the pair part's row sums vanish, plus the data weight
+    for (int idx = c.tid; idx < p * p; idx += c.nt) {
+      const int ra = idx / p, rb = idx - ra * p;
+      const int i = s.grp[ra];
+      if (s.grp[rb] != i) continue;
+      double acc = 0.0;
+      for (int q = 0; q < p; ++q) if (s.grp[q] != i) acc -= s.M[ra * ld + q];
+      s.M[ra * ld + rb] = acc * s.ginv[i] + ((ra == rb) ? s.w[ra] : 0.0);
+    }
+  }
+  return block_sum(c, s, part);
+}
+
 struct Outputs {
   double* A;          // p x m or null
   float* c;           // p or null
@@ -427,19 +517,21 @@ struct Outputs {
   int* status;        // or null
 };
 
-FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int iters) {
+FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int iters, int nweights) {
   for (int i = c.tid; i < p * m; i += c.nt) if (o.A) o.A[i] = 0.0;
-  for (int i = c.tid; i < p; i += c.nt) { if (o.c) o.c[i] = 0.f; if (o.w) o.w[i] = 0.0; }
+  for (int i = c.tid; i < p; i += c.nt) if (o.c) o.c[i] = 0.f;
+  for (int i = c.tid; i < nweights; i += c.nt) if (o.w) o.w[i] = 0.0;
   for (int i = c.tid; i < iters; i += c.nt) if (o.obj) o.obj[i] = 0.0;
   for (int i = c.tid; i < p * p; i += c.nt) if (o.S) o.S[i] = 0.0;
 }
 
 // K: p x p inner products (global or shared memory).  start_from_A: take the subspace in o.A as
 // the current one for the first reweighting (single-step interface); otherwise round one is
-// uniform.  Returns the status bits (same value in every thread).
+// uniform.  nw > 0: the p rows belong to nw workers, cnt[i] consecutive rows each (o.w then has nw
+// entries); nw = 0: one gradient per worker.  Returns the status bits (same value in every thread).
 template <bool LARGE>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
-              bool start_from_A, const Outputs& o) {
+              bool start_from_A, const Outputs& o, int nw = 0, const unsigned char* cnt = nullptr) {
   const int ld = s.ld;
   const int pp = (p + 1) & ~1;
   int status = 0;
@@ -457,7 +549,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   }
   c.sync();
   if (s.flags[1]) {
-    write_zero_outputs(c, o, p, m, iters);
+    write_zero_outputs(c, o, p, m, iters, nw > 0 ? nw : p);
     return ST_NONFINITE;
   }
   for (int i = c.tid; i < p; i += c.nt) s.kd[i] = s.T[i * ld + i];
@@ -465,7 +557,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   double kmax = 0.0;
   for (int i = 0; i < p; ++i) kmax = fmax(kmax, s.kd[i]);
   if (!(kmax > 0.0)) {
-    write_zero_outputs(c, o, p, m, iters);
+    write_zero_outputs(c, o, p, m, iters, nw > 0 ? nw : p);
     return ST_RANK0;
   }
   for (int i = c.tid; i < p; i += c.nt)
@@ -551,11 +643,33 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   }
   c.sync();
 
-  const double coef = (lambda > 0.0 && p > 1) ? lambda / (double)(p - 1) : 0.0;
+  const bool grouped = nw > 0;
+  const int workers = grouped ? nw : p;
+  if (grouped) {
+    if (c.tid == 0) {
+      int row = 0;
+      for (int i = 0; i < nw; ++i) {
+        s.first[i] = row;
+        s.ginv[i] = 1.0 / (double)cnt[i];
+        for (int q = 0; q < (int)cnt[i]; ++q) s.grp[row++] = i;
+      }
+    }
+    c.sync();
+    for (int i = c.tid; i < nw; i += c.nt) {
+      const int r0 = s.first[i], r1 = (i + 1 < nw) ? s.first[i + 1] : p;
+      double acc = 0.0;
+      for (int row = r0; row < r1; ++row) acc += s.fn[row];
+      s.gtr[i] = acc;
+    }
+    c.sync();
+    s.nw = nw;
+  }
+  const double coef = (lambda > 0.0 && workers > 1) ? lambda / (double)(workers - 1) : 0.0;
 
   // ---- weights of the first round
   if (!start_from_A) {
-    (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
+    if (grouped) (void)weights_and_objective_grouped(c, s, s.P, 0, r, p, coef, true, a);
+    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
   } else {
     // Z0 = F A (r x m) -> J buffer; C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
     for (int idx = c.tid; idx < r * m; idx += c.nt) {
@@ -579,12 +693,14 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       s.tmp[k * ld + i] = acc;
     }
     c.sync();
-    (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a);
+    if (grouped) (void)weights_and_objective_grouped(c, s, s.tmp, 0, r, p, coef, false, a);
+    else (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a);
   }
 
   int m_eff = 0;
   for (int t = 0; t < iters; ++t) {
     for (int i = c.tid; i < p; i += c.nt) s.wused[i] = s.w[i];
+    if (grouped) for (int i = c.tid; i < nw; i += c.nt) s.gwused[i] = s.gw[i];
     // ---- T = P M P^T (current basis)
     if (coef > 0.0) {
       for (int idx = c.tid; idx < p * r; idx += c.nt) {       // tmp[i][a] = sum_j M[i][j] P[a][j]
@@ -640,7 +756,8 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
 
     // ---- terms of Eq. (5) at the new subspace, and the next round's weights
-    double obj = weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a);
+    double obj = grouped ? weights_and_objective_grouped(c, s, s.P, m_eff, r, p, coef, false, a)
+                         : weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
   }
   if (m_eff < m) status |= ST_RANK_LT_M;
@@ -652,7 +769,10 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       o.A[idx] = (q < m_eff) ? s.Aacc[i * ld + q] : 0.0;
     }
   }
-  if (o.w) for (int i = c.tid; i < p; i += c.nt) o.w[i] = s.wused[i];
+  if (o.w) {
+    if (grouped) for (int i = c.tid; i < nw; i += c.nt) o.w[i] = s.gwused[i];
+    else for (int i = c.tid; i < p; i += c.nt) o.w[i] = s.wused[i];
+  }
   if (o.S) {   // Y Y^T G = G S with S = A (A^T K): (A^T K) e_j are the leading coordinates of f_j
     for (int idx = c.tid; idx < p * p; idx += c.nt) {
       const int i = idx / p, j = idx - i * p;
@@ -664,14 +784,15 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   if (o.c) {
     for (int k = c.tid; k < m_eff; k += c.nt) {        // s_k = sum_j P[k][j]  (Z^T F 1)
       double acc = 0.0;
-      for (int j = 0; j < p; ++j) acc += s.P[k * ld + j];
+      if (grouped) for (int j = 0; j < p; ++j) acc += s.P[k * ld + j] * s.ginv[s.grp[j]];   // sum of worker means
+      else for (int j = 0; j < p; ++j) acc += s.P[k * ld + j];
       s.ev[k] = acc;
     }
     c.sync();
     for (int i = c.tid; i < p; i += c.nt) {
       double acc = 0.0;
       for (int k = 0; k < m_eff; ++k) acc += s.Aacc[i * ld + k] * s.ev[k];
-      o.c[i] = (float)(acc / (double)p);
+      o.c[i] = (float)(acc / (double)workers);
     }
   }
   return status;

@@ -32,6 +32,8 @@ struct IrlsArgs {
   double* obj;
   double* S;         // p x p selection matrix or null
   int* status;
+  int workers;               // > 0: the p rows belong to this many workers, counts[i] consecutive rows each
+  unsigned char counts[64];  //      (w then has `workers` entries); 0: one gradient per worker
 };
 cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st);
 

@@ -10,6 +10,7 @@ import pytest
 import torch
 
 import synthetic_inputs as si
+from oracle import fa_multi as fm
 from oracle import fa_oracle as fo
 
 pytestmark = pytest.mark.gpu
@@ -178,6 +179,76 @@ def test_aggregate_ex_equals_its_parts(fa):
         fa.fa_aggregate_ex(G, 8, 0.01, 1.0, 7)
     with pytest.raises(fa.FaError):
         fa.fa_irls_ex(torch.eye(3, dtype=torch.float64, device="cuda"), 2, 0.0, float("nan"), 3)
+
+
+def _worker_rows(counts, n, seed, outliers, bf16=False):
+    """Rows of workers with counts[i] gradients each: a common mean, a per-worker offset, per-gradient noise;
+    the last `outliers` workers send large random gradients."""
+    r = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, len(counts), n, 91])))
+    mu = r.standard_normal(n).astype(np.float32)
+    rows = []
+    for i, k in enumerate(counts):
+        if i >= len(counts) - outliers:
+            block = np.float32(5.0) * r.standard_normal((k, n)).astype(np.float32)
+        else:
+            centre = mu + np.float32(0.2) * r.standard_normal(n).astype(np.float32)
+            block = centre[None, :] + np.float32(0.5) * r.standard_normal((k, n)).astype(np.float32)
+        rows.append(block)
+    G = np.ascontiguousarray(np.concatenate(rows, axis=0), dtype=np.float32)
+    return si.f32_to_bf16_bits(G) if bf16 else G
+
+
+MULTI_IRLS = [
+    ([1] * 9, 40, 4, 0.3, 2.0, 7, 2), ([3, 1, 2, 4, 1], 200, 3, 0.0, 2.0, 8, 1), ([3, 1, 2, 4, 1], 200, 5, 0.4, 2.0, 8, 1),
+    ([2, 3, 1, 4, 2, 1, 3], 300, 6, 0.5, 3.0, 10, 2), ([4] * 16, 500, 20, 0.05, 2.0, 8, 3), ([1, 63], 100, 3, 0.2, 2.0, 5, 0),
+    ([5], 50, 2, 0.3, 2.0, 4, 0), ([2] * 15, 1000, 8, 0.01, 2.0, 10, 3), ([8, 7, 8, 8], 400, 10, 0.1, 1.5, 6, 1),
+]
+
+
+@pytest.mark.parametrize("counts,n,m,lam,a,iters,outliers", MULTI_IRLS)
+def test_irls_for_workers_with_several_gradients(fa, counts, n, m, lam, a, iters, outliers):
+    G = _worker_rows(counts, n, 3, outliers).astype(np.float64)
+    ref = fm.fa_aggregate_multi(G, counts, m, lam, iters, a=a)
+    rows, nw = G.shape[0], len(counts)
+    K = torch.from_numpy(fo.inner_products(G)).cuda()
+    A = torch.zeros((rows, m), dtype=torch.float64, device="cuda")
+    w = torch.full((nw + 2,), float("nan"), dtype=torch.float64, device="cuda")
+    obj = torch.zeros(iters, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = fa.fa_irls_multi(K, counts, m, lam, iters, a=a, A_out=A, w_out=w, obj_out=obj, status=status)
+    torch.cuda.synchronize()
+    k = ref["Y"].shape[1]
+    assert int(status.item()) & ~fa.ST_RANK_LT_M == 0
+    assert torch.isnan(w[nw:]).all()                     # one weight per worker, nothing written beyond
+    Y = G.T @ A.cpu().numpy()[:, :k]
+    assert np.abs(Y.T @ Y - np.eye(k)).max() < 1e-9
+    assert fo.principal_angles(ref["Y"], Y).max() < 1e-7
+    assert np.allclose(obj.cpu().numpy(), ref["objective"], rtol=1e-9, atol=1e-9)
+    assert np.allclose(w[:nw].cpu().numpy(), ref["w"], rtol=1e-6, atol=0)
+    assert fo.rel_l2(c.cpu().numpy().astype(np.float64) @ G, ref["d"]) < 1e-6
+
+
+MULTI_AGG = [
+    ([3, 1, 2, 4, 1], 70_001, False, 4, 0.2, 2.0, 7, 1), ([2] * 15, 50_000, False, 8, 0.01, 2.0, 8, 3),
+    ([4] * 16, 66_000, True, 16, 0.02, 2.0, 6, 3), ([1] * 15, 65_537, False, 8, 0.01, 3.0, 6, 2),
+]
+
+
+@pytest.mark.parametrize("counts,n,bf16,m,lam,a,iters,outliers", MULTI_AGG)
+def test_aggregate_for_workers_with_several_gradients(fa, counts, n, bf16, m, lam, a, iters, outliers):
+    from tests.gpu_util import to_device
+    G_np = _worker_rows(counts, n, 8, outliers, bf16=bf16)
+    G, _ = to_device(G_np)
+    out = fa.fa_aggregate_multi(G, counts, m, lam, iters, a=a)
+    torch.cuda.synchronize()
+    ref = fm.fa_aggregate_multi(si.to_float64(G_np), counts, m, lam, iters, a=a)
+    rel_tol, _ = TOL["bf16" if bf16 else "f32"]
+    assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < rel_tol
+    if all(k == 1 for k in counts):
+        assert torch.equal(out, fa.fa_aggregate_ex(G, m, lam, a, iters))
+    for bad in ([1] * (len(counts) - 1), [0] + list(counts), list(counts) + [1]):
+        with pytest.raises(fa.FaError):
+            fa.fa_aggregate_multi(G, bad, m, lam, iters)
 
 
 def _aggregate_and_compare(fa, G_np, m, lam, iters, dtype_key, mis=0):
