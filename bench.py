@@ -177,6 +177,9 @@ def main():
     ap.add_argument("--buffers", type=int, default=3, help="independent copies of G rotated between steps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="N > 1: split the ONE workload along n over the ranks (partial inner products summed by an "
+                         "all-reduce of p*p doubles per step) instead of running N replicas; strong scaling")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -209,6 +212,13 @@ def main():
     # step never finds its gradients in L2 from the previous step); every copy is > L2 at cfg2
     G_np = si.generate(w)
     host = torch.from_numpy(G_np.view(np.int16)).view(torch.bfloat16) if w.dtype == "bf16" else torch.from_numpy(G_np)
+    sharded_mode = args.sharded and world > 1
+    n_total = w.n
+    if sharded_mode:                       # this rank keeps its columns only; everything below sees the shard
+        from paper_2302_05865_b200 import sharded
+        lo, hi = sharded.shard_bounds(w.n, world, rank)
+        host = host[:, lo:hi].contiguous()
+        w = w.scaled(hi - lo)
     nbuf = max(1, args.buffers)
     Gs = [host.cuda() for _ in range(nbuf)]
     out = torch.empty(w.n, dtype=torch.float32, device="cuda")
@@ -216,8 +226,14 @@ def main():
     wsb = fa.new_workspace(Gs[0], w.m)
     stream = torch.cuda.current_stream()
 
-    def step(i):
-        fa.fa_aggregate(Gs[i % nbuf], w.m, w.lam, w.iters, out=out, ws=wsb, status=status, stream=stream)
+    if sharded_mode:
+        sharded_step = sharded.ShardedStep(w.m, w.lam, w.iters)
+
+        def step(i):
+            sharded_step(Gs[i % nbuf], out=out)
+    else:
+        def step(i):
+            fa.fa_aggregate(Gs[i % nbuf], w.m, w.lam, w.iters, out=out, ws=wsb, status=status, stream=stream)
 
     for i in range(args.warmup):
         step(i)
@@ -244,7 +260,7 @@ def main():
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         elapsed_ms = float(t.item())
     ms_per_step = elapsed_ms / args.steps
-    value = whole_job_rate(elapsed_ms, args.steps, world)
+    value = whole_job_rate(elapsed_ms, args.steps, 1 if sharded_mode else world)
 
     # ---- per-kernel times, same buffers and stream, CUDA events around single launches
     def time_call(fn, reps):
@@ -278,7 +294,7 @@ def main():
 
     # ---- end to end through the host-buffer entry point (pinned host memory both ways)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sharded_mode:
         Gh = host.pin_memory()
         outh = torch.empty(w.n, dtype=torch.float32).pin_memory()
         sth = torch.zeros(1, dtype=torch.int32).pin_memory()
@@ -316,11 +332,13 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
-        "config": {"workload": w.name, "p": w.p, "f": w.f, "n": w.n, "m": w.m, "lambda": w.lam, "iters": w.iters,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if sharded_mode else "weak",
+        "vs_baseline": None, "dtype": "f32" if w.dtype == "f32" else "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "p": w.p, "f": w.f, "n": n_total, "m": w.m, "lambda": w.lam, "iters": w.iters,
                    "storage": w.dtype, "l2": f"inputs larger than L2; {nbuf} device copies of G rotated between steps",
-                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU"},
+                   "parallelism": (f"n-sharded x{world}, one all-reduce of p*p fp64 per step; roofline and kernel "
+                                   f"times are rank 0's shard of {w.n} columns") if sharded_mode
+                                  else (f"replicas x{world}" if world > 1 else "single GPU")},
         "roofline": {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
                      "unit": "GB/s", "frac": gram_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_launch": int(gram_bytes), "ms_per_launch": t_gram},

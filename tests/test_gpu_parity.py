@@ -352,3 +352,30 @@ def test_host_buffer_entry_point_round_trips(fa):
     torch.cuda.synchronize()
     ref = fa.fa_aggregate(torch.from_numpy(G_np).cuda(), w.m, w.lam, w.iters)
     assert torch.equal(outh.cuda(), ref) and int(sth.item()) == 0
+
+
+@pytest.mark.parametrize("p,n,bf16,world", [(15, 300_007, False, 3), (31, 200_000, True, 4), (15, 20, False, 8)])
+def test_column_sharded_step_equals_the_whole_step(fa, p, n, bf16, world):
+    """One GPU plays the ranks one after another (no rank waits on another): pass 1 takes every shard's
+    partial inner products, pass 2 hands each rank the sum in place of the all-reduce."""
+    from paper_2302_05865_b200 import sharded
+    from tests.gpu_util import to_device
+    m, lam, iters = min(8, p), 0.01, 8
+    G_np = si.ladder_case(p, n, 31, "noisy_mean", bf16=bf16)
+    G, _ = to_device(G_np)
+    bounds = [sharded.shard_bounds(n, world, r) for r in range(world)]
+    shards = [G[:, lo:hi].contiguous() for lo, hi in bounds]
+    Ksum = torch.zeros((p, p), dtype=torch.float64, device="cuda")
+    for sh in shards:
+        if sh.shape[1]:
+            Ksum += fa.fa_gram(sh)
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    for (lo, hi), sh in zip(bounds, shards):
+        step = sharded.ShardedStep(m, lam, iters, reduce_fn=lambda K: K.copy_(Ksum))
+        out[lo:hi] = step(sh)
+    torch.cuda.synchronize()
+    ref = fo.fa_aggregate(si.to_float64(G_np), m, lam, iters)
+    rel_tol, _ = TOL["bf16" if bf16 else "f32"]
+    assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < rel_tol
+    whole = fa.fa_aggregate(G, m, lam, iters)
+    assert fo.rel_l2(out.cpu().numpy(), whole.cpu().numpy().astype(np.float64)) < rel_tol
