@@ -35,7 +35,7 @@ formula; this is the reading used, each item listed in the design notes):
   * sqrt(.) in a weight is floored at EPS; zero gradients and identical pairs
     carry weight 0 and contribute 0 to the objective; eigen-directions whose
     eigenvalue is <= RANK_REL * largest are left out of Y;
-  * exactly `iters` rounds are run (no early exit).
+  * exactly `iters` rounds are run unless a tolerance is given (see fa_aggregate).
 
 Two ways of getting the eigenvectors of C are provided and tested against
 each other: "literal" builds the n x n matrix C term by term (small n only);
@@ -209,15 +209,21 @@ def weighted_pca_svd(G, w, W, m):
 
 # -- the iteration -------------------------------------------------------------
 
-def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a=2.0):
+def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a=2.0, Y0=None, tol=None):
     """Run `iters` IRLS rounds and return the aggregate.
 
     G      : (p, n) array, rows are worker gradients (converted to float64)
     a      : surrogate constant of Eq. (4), a > 1; terms are (1 - v)^(1/a) and the reweighting
              of a term with value u is 1 / (normaliser * max(u^(1 - 1/a), eps))  (a = 2: the paper's
              square roots)
+    Y0     : optional (n, k) matrix of full column rank, a subspace to start from (the "smart
+             initialization" Section 2.1 mentions): round one then reweights by the term values at
+             span(Y0) instead of being uniform.  A Y0 of rank 0 (or None) is the cold start.
+    tol    : optional; stop after round t >= 2 once |objective_{t-1} - objective_t| <= tol (the
+             "small error" convergence criterion of the implementation details in Section 3,
+             which the paper pairs with a cap on the rounds: `iters` is that cap)
     returns: dict with d (n,), Y (n, k<=m), u (p,), w (p,) last data weights,
-             objective (list, one per round), evals (last round, descending),
+             objective (list, one per round run), rounds, evals (last round, descending),
              and with history=True the list of Y per round.
     """
     G = np.asarray(G, dtype=np.float64)
@@ -233,15 +239,22 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
 
     if np.all(zero):                       # every gradient is zero: nothing to span
         return dict(d=np.zeros(n), Y=np.zeros((n, 0)), u=np.zeros(p), w=np.zeros(p),
-                    objective=[0.0] * iters, evals=np.zeros(p), Ys=[])
+                    objective=[0.0] * iters, rounds=iters, evals=np.zeros(p), Ys=[])
 
     u = np.zeros(p)
     U = np.zeros((p, p))
+    warm = False
+    if Y0 is not None and np.asarray(Y0).size:
+        Q, R = np.linalg.qr(np.asarray(Y0, dtype=np.float64))
+        diag = np.abs(np.diag(R))
+        if diag.size and diag.min() > 1e-12 * diag.max():
+            u, U = term_values(G, Q, lam, norms, zero, D2, active)
+            warm = True
     objs, Ys = [], []
     for t in range(1, iters + 1):
         w = np.zeros(p)
         W = np.zeros((p, p))
-        if t == 1:
+        if t == 1 and not warm:
             w[~zero] = 1.0
             W[active] = coef
         else:
@@ -258,8 +271,10 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
         objs.append(obj)
         if history:
             Ys.append(Y)
+        if tol is not None and t >= 2 and abs(objs[-2] - objs[-1]) <= tol:
+            break
     d = Y @ (Y.T @ G.sum(axis=0)) / p
-    return dict(d=d, Y=Y, u=u, w=w, objective=objs, evals=evals, Ys=Ys)
+    return dict(d=d, Y=Y, u=u, w=w, objective=objs, rounds=len(objs), evals=evals, Ys=Ys)
 
 
 def reconstruction(G, Y):

@@ -434,3 +434,53 @@ def test_reconstruction_is_the_orthogonal_projection():
     assert np.allclose(R, G @ P, atol=1e-12)
     assert np.allclose(R.mean(axis=0), out["d"], atol=1e-12)          # its column average is the update
     assert np.allclose((G - R) @ out["Y"], 0.0, atol=1e-10)           # residuals are orthogonal to Y
+
+
+# ---- start from a given subspace, stop on a tolerance --------------------------------------------
+
+@pytest.mark.parametrize("lam", [0.0, 0.3])
+def test_start_from_the_pca_subspace_is_the_cold_start_shifted_by_one_round(lam):
+    """Round one of the cold start is PCA; starting from that subspace, round t is cold round t + 1."""
+    G = noisy_mean(9, 30, 50, sigma=0.5, outliers=2, scale_spread=True)
+    cold = fo.fa_aggregate(G, 3, lam, iters=6, history=True)
+    _, _, Vt = np.linalg.svd(G, full_matrices=False)              # PCA of the gradient matrix, by SVD of G itself
+    Ypca = Vt[:3].T
+    if lam > 0:
+        Ypca = cold["Ys"][0]                                      # with the regulariser round one is not plain PCA
+    warm = fo.fa_aggregate(G, 3, lam, iters=5, Y0=Ypca, history=True)
+    for t in range(5):
+        assert fo.principal_angles(cold["Ys"][t + 1], warm["Ys"][t]).max() < 1e-9
+    assert np.allclose(cold["objective"][1:], warm["objective"], rtol=1e-10)
+
+
+def test_start_depends_on_the_span_only_and_the_fixed_point_stays():
+    G = noisy_mean(8, 25, 51, sigma=0.5, outliers=1)
+    Y0 = rng(52).standard_normal((25, 3))
+    mix = rng(53).standard_normal((3, 3)) + 3 * np.eye(3)
+    a = fo.fa_aggregate(G, 3, 0.2, iters=4, Y0=Y0)
+    b = fo.fa_aggregate(G, 3, 0.2, iters=4, Y0=Y0 @ mix)
+    assert fo.principal_angles(a["Y"], b["Y"]).max() < 1e-9
+    star = fo.fa_aggregate(G, 3, 0.2, iters=400)
+    again = fo.fa_aggregate(G, 3, 0.2, iters=1, Y0=star["Y"])
+    assert fo.principal_angles(star["Y"], again["Y"]).max() < 1e-6
+    assert abs(again["objective"][0] - star["objective"][-1]) < 1e-9
+    # a start of rank 0 is the cold start
+    cold = fo.fa_aggregate(G, 3, 0.2, iters=3)
+    zero = fo.fa_aggregate(G, 3, 0.2, iters=3, Y0=np.zeros((25, 3)))
+    assert np.allclose(cold["objective"], zero["objective"], rtol=0, atol=0)
+
+
+def test_tolerance_stops_at_the_first_small_decrease_and_not_before():
+    G = noisy_mean(10, 40, 54, sigma=0.5, outliers=2)
+    full = fo.fa_aggregate(G, 4, 0.1, iters=60)["objective"]
+    steps = np.abs(np.diff(full))
+    tol = 1e-6
+    first = int(np.nonzero(steps <= tol)[0][0]) + 2               # rounds run when the test first succeeds
+    out = fo.fa_aggregate(G, 4, 0.1, iters=60, tol=tol)
+    assert out["rounds"] == first and len(out["objective"]) == first
+    assert np.array_equal(out["objective"], full[:first])
+    same = fo.fa_aggregate(G, 4, 0.1, iters=first)
+    assert fo.principal_angles(same["Y"], out["Y"]).max() < 1e-12 and fo.rel_l2(out["d"], same["d"]) < 1e-12
+    assert fo.fa_aggregate(G, 4, 0.1, iters=7, tol=0.0)["rounds"] == 7       # the cap
+    assert fo.fa_aggregate(G, 4, 0.1, iters=7, tol=1e9)["rounds"] == 2
+    assert fo.fa_aggregate(G, 4, 0.1, iters=1, tol=1e9)["rounds"] == 1
