@@ -121,6 +121,24 @@ int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double 
                     int iters, float* out, double* A_out, double* S_out, void* ws, size_t ws_bytes,
                     int* status, void* stream);
 
+/* IRLS that starts from a given subspace and may stop early.
+ *   A0   : p x m fp64 row-major or NULL.  The first reweighting uses the term values at span(G^T A0)
+ *          instead of uniform weights (the "smart initialization" Section 2.1 mentions): pass the
+ *          A_out of the previous training step to continue from its subspace with fewer rounds.
+ *          Any full-rank A0 will do (its image is orthonormalised on the device); a rank-deficient or
+ *          zero A0, and NULL, give the uniform first round.  A0 may be the same buffer as A_out.
+ *   tol  : >= 0: stop after round t >= 2 once |objective_{t-1} - objective_t| <= tol (the
+ *          small-error convergence criterion of Section 3, implementation details), iters being
+ *          the cap on the rounds; < 0: run all iters rounds.  NaN is an argument error.
+ *   rounds_out : out, device int or NULL: rounds run.  Entries of obj_out past it repeat the last value. */
+int fa_irls_warm(const double* K, int p, int m, double lambda, double a, int iters, double tol,
+                 const double* A0, double* A_out, float* c_out, double* w_out, double* obj_out,
+                 int* rounds_out, int* status, void* stream);
+
+int fa_aggregate_warm(const void* G, int dtype, int p, long long n, int m, double lambda, double a,
+                      int iters, double tol, const double* A0, float* out, double* A_out,
+                      int* rounds_out, void* ws, size_t ws_bytes, int* status, void* stream);
+
 /* Workers that hand in several gradients each (Section 2.1, "Advantages of Subspace based Aggregation";
  * the extension paragraph of Section 2.2; the appendix restatement of Eq. (5) with
  * tr(Y^T g_i g_i^T Y) / tr(g_i^T g_i)).  The `rows` gradients are the rows of G as before, the

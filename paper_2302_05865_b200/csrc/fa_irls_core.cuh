@@ -515,6 +515,7 @@ struct Outputs {
   double* obj;        // iters (or 1) or null
   double* S;          // p x p selection matrix or null
   int* status;        // or null
+  int* rounds;        // rounds actually run, or null
 };
 
 FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int iters, int nweights) {
@@ -523,15 +524,20 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
   for (int i = c.tid; i < nweights; i += c.nt) if (o.w) o.w[i] = 0.0;
   for (int i = c.tid; i < iters; i += c.nt) if (o.obj) o.obj[i] = 0.0;
   for (int i = c.tid; i < p * p; i += c.nt) if (o.S) o.S[i] = 0.0;
+  if (o.rounds && c.tid == 0) *o.rounds = 0;
 }
 
-// K: p x p inner products (global or shared memory).  start_from_A: take the subspace in o.A as
-// the current one for the first reweighting (single-step interface); otherwise round one is
-// uniform.  nw > 0: the p rows belong to nw workers, cnt[i] consecutive rows each (o.w then has nw
+// K: p x p inner products (global or shared memory).  start: 0 = round one is uniform; 1 = take the
+// subspace spanned by G^T A0 as the current one for the first reweighting, A0 being the A of an
+// earlier round on the same K (its image is orthonormal already: single-step interface); 2 = the
+// same for any A0 (p x m), e.g. the A of the previous training step: its image is orthonormalised
+// first, and a rank-deficient one falls back to the uniform round.  tol >= 0: stop after round
+// t >= 2 once the objective moved by <= tol (remaining entries of o.obj repeat the last value).  nw > 0: the p rows belong to nw workers, cnt[i] consecutive rows each (o.w then has nw
 // entries); nw = 0: one gradient per worker.  Returns the status bits (same value in every thread).
 template <bool LARGE>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
-              bool start_from_A, const Outputs& o, int nw = 0, const unsigned char* cnt = nullptr) {
+              int start, const double* A0, double tol, const Outputs& o, int nw = 0,
+              const unsigned char* cnt = nullptr) {
   const int ld = s.ld;
   const int pp = (p + 1) & ~1;
   int status = 0;
@@ -667,18 +673,61 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   const double coef = (lambda > 0.0 && workers > 1) ? lambda / (double)(workers - 1) : 0.0;
 
   // ---- weights of the first round
-  if (!start_from_A) {
-    if (grouped) (void)weights_and_objective_grouped(c, s, s.P, 0, r, p, coef, true, a);
-    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
-  } else {
-    // Z0 = F A (r x m) -> J buffer; C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
+  if (start != 0) {
+    // Z0 = F A0 (r x m) -> J buffer
     for (int idx = c.tid; idx < r * m; idx += c.nt) {
       int k = idx / m, q = idx - k * m;
       double acc = 0.0;
-      for (int i = 0; i < p; ++i) acc += s.P[k * ld + i] * o.A[i * m + q];
+      for (int i = 0; i < p; ++i) acc += s.P[k * ld + i] * A0[i * m + q];
       s.J[k * ld + q] = acc;
     }
     c.sync();
+    if (start == 2) {
+      // W = Z0^T Z0 -> T; Cholesky W = L L^T by one thread; Z = Z0 L^-T row by row
+      for (int idx = c.tid; idx < m * m; idx += c.nt) {
+        int q = idx / m, l = idx - q * m;
+        double acc = 0.0;
+        for (int k = 0; k < r; ++k) acc += s.J[k * ld + q] * s.J[k * ld + l];
+        s.T[q * ld + l] = acc;
+      }
+      c.sync();
+      if (c.tid == 0) {
+        double dmin = 1.7e308, dmax = 0.0;
+        bool ok = true;
+        for (int q = 0; q < m && ok; ++q) {
+          double d = s.T[q * ld + q];
+          for (int l = 0; l < q; ++l) d -= s.T[q * ld + l] * s.T[q * ld + l];
+          if (!(d > 0.0)) { ok = false; break; }
+          const double lqq = sqrt(d);
+          s.T[q * ld + q] = lqq;
+          dmin = fmin(dmin, lqq); dmax = fmax(dmax, lqq);
+          for (int i = q + 1; i < m; ++i) {
+            double v = s.T[i * ld + q];
+            for (int l = 0; l < q; ++l) v -= s.T[i * ld + l] * s.T[q * ld + l];
+            s.T[i * ld + q] = v / lqq;
+          }
+        }
+        s.flags[1] = (ok && dmin > 1e-12 * dmax) ? 1 : 0;
+      }
+      c.sync();
+      if (s.flags[1] == 0) start = 0;
+      else {
+        for (int k = c.tid; k < r; k += c.nt) {
+          for (int q = 0; q < m; ++q) {
+            double v = s.J[k * ld + q];
+            for (int l = 0; l < q; ++l) v -= s.J[k * ld + l] * s.T[q * ld + l];
+            s.J[k * ld + q] = v / s.T[q * ld + q];
+          }
+        }
+      }
+      c.sync();
+    }
+  }
+  if (start == 0) {
+    if (grouped) (void)weights_and_objective_grouped(c, s, s.P, 0, r, p, coef, true, a);
+    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
+  } else {
+    // C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
     for (int idx = c.tid; idx < m * p; idx += c.nt) {
       int q = idx / p, i = idx - q * p;
       double acc = 0.0;
@@ -697,7 +746,8 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     else (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a);
   }
 
-  int m_eff = 0;
+  int m_eff = 0, rounds = iters;
+  double prev_obj = 0.0;
   for (int t = 0; t < iters; ++t) {
     for (int i = c.tid; i < p; i += c.nt) s.wused[i] = s.w[i];
     if (grouped) for (int i = c.tid; i < nw; i += c.nt) s.gwused[i] = s.gw[i];
@@ -759,7 +809,14 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     double obj = grouped ? weights_and_objective_grouped(c, s, s.P, m_eff, r, p, coef, false, a)
                          : weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
+    if (tol >= 0.0 && t >= 1 && fabs(prev_obj - obj) <= tol) {      // same value in every thread
+      rounds = t + 1;
+      if (o.obj) for (int q = t + 1 + c.tid; q < iters; q += c.nt) o.obj[q] = obj;
+      break;
+    }
+    prev_obj = obj;
   }
+  if (o.rounds && c.tid == 0) *o.rounds = rounds;
   if (m_eff < m) status |= ST_RANK_LT_M;
 
   // ---- outputs

@@ -25,7 +25,10 @@ struct IrlsArgs {
   int p, m, iters;
   double lambda;
   double a;          // surrogate constant of Eq. (4); 2 = the paper's square roots
-  int start_from_A;
+  int start_from_A;  // 0 uniform first round; 1 start from A0 (orthonormal image); 2 start from any A0
+  const double* A0;  // p x m, read before A is written (may alias A)
+  double tol;        // >= 0: stop once the objective moved by <= tol; < 0: run all rounds
+  int* rounds;       // rounds run, or null
   double* A;
   float* c;
   double* w;

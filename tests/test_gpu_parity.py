@@ -379,3 +379,62 @@ def test_column_sharded_step_equals_the_whole_step(fa, p, n, bf16, world):
     assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < rel_tol
     whole = fa.fa_aggregate(G, m, lam, iters)
     assert fo.rel_l2(out.cpu().numpy(), whole.cpu().numpy().astype(np.float64)) < rel_tol
+
+
+WARM_CASES = [(15, 2000, "noisy_mean", 8, 0.01, 6), (7, 33, "dup_zero", 3, 0.2, 5), (31, 3000, "noisy_mean", 12, 0.01, 6),
+              (64, 300, "noisy_mean", 20, 0.01, 5), (2, 5, "noisy_mean", 1, 0.3, 4)]
+
+
+@pytest.mark.parametrize("p,n,kind,m,lam,iters", WARM_CASES)
+def test_irls_from_a_given_subspace_and_with_a_tolerance(fa, p, n, kind, m, lam, iters):
+    G = si.ladder_case(p, n, 9, kind).astype(np.float64)
+    K = torch.from_numpy(fo.inner_products(G)).cuda()
+    A0_np = np.random.default_rng(1).standard_normal((p, m))
+    A = torch.from_numpy(A0_np).cuda()                          # started from and overwritten in place
+    obj = torch.zeros(iters, dtype=torch.float64, device="cuda")
+    rounds = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = fa.fa_irls_warm(K, m, lam, iters, A0=A, A_out=A, obj_out=obj, rounds_out=rounds)
+    ref = fo.fa_aggregate(G, m, lam, iters, Y0=G.T @ A0_np)
+    k = ref["Y"].shape[1]
+    assert int(rounds.item()) == iters
+    assert fo.principal_angles(ref["Y"], G.T @ A.cpu().numpy()[:, :k]).max() < 1e-7
+    assert np.allclose(obj.cpu().numpy(), ref["objective"], rtol=1e-9, atol=1e-9)
+    assert fo.rel_l2(c.cpu().numpy().astype(np.float64) @ G, ref["d"]) < 1e-6
+    # a start without rank is the uniform first round
+    cold = fa.fa_irls(K, m, lam, iters)
+    zero = fa.fa_irls_warm(K, m, lam, iters, A0=torch.zeros((p, m), dtype=torch.float64, device="cuda"))
+    assert torch.equal(cold, zero) and torch.equal(cold, fa.fa_irls_warm(K, m, lam, iters))
+    # tolerance: same number of rounds as the oracle, same result, tail of the objective repeated
+    cap, tol = 40, 1e-5
+    ref = fo.fa_aggregate(G, m, lam, cap, tol=tol)
+    obj = torch.full((cap,), float("nan"), dtype=torch.float64, device="cuda")
+    c = fa.fa_irls_warm(K, m, lam, cap, tol=tol, obj_out=obj, rounds_out=rounds)
+    r = int(rounds.item())
+    oh = obj.cpu().numpy()
+    assert r == ref["rounds"]
+    assert np.allclose(oh[:r], ref["objective"], rtol=1e-9, atol=1e-9) and (oh[r:] == oh[r - 1]).all()
+    assert fo.rel_l2(c.cpu().numpy().astype(np.float64) @ G, ref["d"]) < 1e-6
+
+
+def test_aggregate_continues_from_the_previous_steps_subspace(fa):
+    """Two training steps: the second starts from the first one's A and needs fewer rounds."""
+    from tests.gpu_util import to_device
+    p, n, m, lam = 15, 120_001, 8, 0.01
+    G1_np = si.ladder_case(p, n, 41, "noisy_mean")
+    noise = np.random.Generator(np.random.PCG64(42)).standard_normal((p, n)).astype(np.float32)
+    G2_np = (G1_np + np.float32(0.05) * noise).astype(np.float32)          # the next step's gradients
+    G1, _ = to_device(G1_np)
+    G2, _ = to_device(G2_np)
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    rounds = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fa.fa_aggregate_warm(G1, m, lam, 30, tol=1e-7, A_out=A, rounds_out=rounds)
+    r_cold = int(rounds.item())
+    A_prev = A.clone()
+    out = fa.fa_aggregate_warm(G2, m, lam, 30, tol=1e-7, A0=A, A_out=A, rounds_out=rounds)
+    r_warm = int(rounds.item())
+    ref = fo.fa_aggregate(G2_np.astype(np.float64), m, lam, 30, tol=1e-7,
+                          Y0=G2_np.astype(np.float64).T @ A_prev.cpu().numpy())
+    assert r_warm == ref["rounds"] and r_warm <= r_cold
+    assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < 1e-4
+    with pytest.raises(fa.FaError):
+        fa.fa_aggregate_warm(G2, m, lam, 5, tol=float("nan"))
