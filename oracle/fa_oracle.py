@@ -191,6 +191,19 @@ def pair_weight_matrix(w, W):
     return M
 
 
+def weighted_pca_qr(G, w, W, m):
+    """Same subspace when some weights are negative (C indefinite): with the thin QR G^T = Q R,
+    C = G^T M G = Q (R M R^T) Q^T, so the eigenvectors of C with non-zero eigenvalue are Q times
+    those of the p x p matrix R M R^T."""
+    M = pair_weight_matrix(w, W)
+    Q, R = np.linalg.qr(G.T)
+    S = R @ M @ R.T
+    evals, V = np.linalg.eigh(0.5 * (S + S.T))
+    evals, V = evals[::-1], V[:, ::-1]
+    k = _keep(evals, min(m, G.shape[1]))
+    return Q @ V[:, :k], evals
+
+
 def weighted_pca_svd(G, w, W, m):
     """Same subspace from the thin SVD of B = G^T M^(1/2) (n x p)."""
     p, n = G.shape
@@ -209,13 +222,25 @@ def weighted_pca_svd(G, w, W, m):
 
 # -- the iteration -------------------------------------------------------------
 
-def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a=2.0, Y0=None, tol=None):
+def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a=2.0, Y0=None, tol=None,
+                 alpha=1.0, beta=0.5):
     """Run `iters` IRLS rounds and return the aggregate.
 
     G      : (p, n) array, rows are worker gradients (converted to float64)
     a      : surrogate constant of Eq. (4), a > 1; terms are (1 - v)^(1/a) and the reweighting
              of a term with value u is 1 / (normaliser * max(u^(1 - 1/a), eps))  (a = 2: the paper's
              square roots)
+    alpha, beta : shape parameters of the Beta likelihood of the values v_i (Eq. (1) uses alpha = 1,
+             beta = 1/2).  The negative log-likelihood -(alpha-1) log v - (beta-1) log(1-v), with
+             the surrogate log x ~ a x^(1/a) - a of Eq. (4) on both logarithms (the "two terms" of the
+             extension paragraph of Section 2.2) and the scale in which alpha = 1, beta = 1/2 gives
+             the data term of Eq. (5), is the data term
+                 2 (1 - beta) (1 - v_i)^(1/a) + 2 (1 - alpha) v_i^(1/a).
+             Both terms are concave in v_i for alpha <= 1, beta <= 1 (required here), so the tangent
+             majoriser gives the weight
+                 [2 (1 - beta) / max(u_i^(1-1/a), eps) - 2 (1 - alpha) / max(v_i^(1-1/a), eps)] / ||g_i||^2,
+             which may be negative; C is then indefinite and only eigen-directions with positive
+             eigenvalue enter Y.
     Y0     : optional (n, k) matrix of full column rank, a subspace to start from (the "smart
              initialization" Section 2.1 mentions): round one then reweights by the term values at
              span(Y0) instead of being uniform.  A Y0 of rank 0 (or None) is the cold start.
@@ -232,16 +257,38 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
         raise ValueError("need 1 <= m <= p")
     if iters < 1 or lam < 0 or not (a > 1.0):
         raise ValueError("need iters >= 1, lam >= 0 and a > 1")
+    if not (0.0 < alpha <= 1.0 and 0.0 < beta <= 1.0):
+        raise ValueError("need 0 < alpha <= 1 and 0 < beta <= 1")
     norms, zero = _classify(G)
     D2, active = _pairs(G, norms, lam)
     coef = lam / (p - 1) if (lam > 0 and p > 1) else 0.0
-    pca = weighted_pca_literal if method == "literal" else weighted_pca_svd
+    cb, ca = 2.0 * (1.0 - beta), 2.0 * (1.0 - alpha)
+    if method == "literal":
+        pca = weighted_pca_literal
+    elif ca != 0.0 or method == "qr":
+        pca = weighted_pca_qr
+    else:
+        pca = weighted_pca_svd
+
+    def explained(Y):
+        """v_i = ||Y^T g_i||^2 / ||g_i||^2 (Section 2.1), 0 for a zero gradient."""
+        Z = G @ Y
+        v = np.zeros(p)
+        v[~zero] = np.einsum("ij,ij->i", Z, Z)[~zero] / norms[~zero]
+        return v
+
+    def data_terms(u, v):
+        t = np.maximum(u, 0.0) ** (1.0 / a) if cb == 1.0 else cb * np.maximum(u, 0.0) ** (1.0 / a)
+        if ca != 0.0:
+            t = t + ca * np.where(zero, 0.0, np.maximum(v, 0.0) ** (1.0 / a))
+        return float(np.sum(t))
 
     if np.all(zero):                       # every gradient is zero: nothing to span
         return dict(d=np.zeros(n), Y=np.zeros((n, 0)), u=np.zeros(p), w=np.zeros(p),
                     objective=[0.0] * iters, rounds=iters, evals=np.zeros(p), Ys=[])
 
     u = np.zeros(p)
+    v = np.zeros(p)
     U = np.zeros((p, p))
     warm = False
     if Y0 is not None and np.asarray(Y0).size:
@@ -249,6 +296,7 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
         diag = np.abs(np.diag(R))
         if diag.size and diag.min() > 1e-12 * diag.max():
             u, U = term_values(G, Q, lam, norms, zero, D2, active)
+            v = explained(Q)
             warm = True
     objs, Ys = [], []
     for t in range(1, iters + 1):
@@ -259,13 +307,18 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
             W[active] = coef
         else:
             r = np.maximum(u, 0.0) ** (1.0 - 1.0 / a)
-            w[~zero] = 1.0 / (norms[~zero] * np.maximum(r[~zero], eps))
+            if cb == 1.0 and ca == 0.0:
+                w[~zero] = 1.0 / (norms[~zero] * np.maximum(r[~zero], eps))
+            else:
+                rv = np.maximum(v, 0.0) ** (1.0 - 1.0 / a)
+                w[~zero] = (cb / np.maximum(r[~zero], eps) - ca / np.maximum(rv[~zero], eps)) / norms[~zero]
             if coef > 0:
                 R = np.maximum(U, 0.0) ** (1.0 - 1.0 / a)
                 W[active] = coef / (D2[active] * np.maximum(R[active], eps))
         Y, evals = pca(G, w, W, m)
         u, U = term_values(G, Y, lam, norms, zero, D2, active)
-        obj = float(np.sum(np.maximum(u, 0.0) ** (1.0 / a)))
+        v = explained(Y)
+        obj = data_terms(u, v)
         if coef > 0:
             obj += coef * float(np.sum(np.maximum(U, 0.0) ** (1.0 / a)))
         objs.append(obj)

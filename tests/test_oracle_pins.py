@@ -484,3 +484,103 @@ def test_tolerance_stops_at_the_first_small_decrease_and_not_before():
     assert fo.fa_aggregate(G, 4, 0.1, iters=7, tol=0.0)["rounds"] == 7       # the cap
     assert fo.fa_aggregate(G, 4, 0.1, iters=7, tol=1e9)["rounds"] == 2
     assert fo.fa_aggregate(G, 4, 0.1, iters=1, tol=1e9)["rounds"] == 1
+
+
+# ---- general Beta(alpha, beta) likelihood of the values (extension paragraph of Section 2.2) ----------
+
+def beta_objective(G, Y, lam, a, alpha, beta):
+    """-(alpha-1) log v - (beta-1) log(1-v) with log x -> a x^(1/a) - a on both logarithms, divided by a/2
+    and without the constants, plus the regulariser of Eq. (5): typed out here with traces."""
+    p = G.shape[0]
+    val = 0.0
+    for i in range(p):
+        x = G[i]
+        if x @ x > 0:
+            v = np.trace(Y.T @ np.outer(x, x) @ Y) / (x @ x)
+            val += 2 * (1 - beta) * max(1.0 - v, 0.0) ** (1 / a) + 2 * (1 - alpha) * max(v, 0.0) ** (1 / a)
+    if lam > 0:
+        for i in range(p):
+            for j in range(p):
+                x = G[i] - G[j]
+                if i != j and x @ x > 0:
+                    v = np.trace(Y.T @ np.outer(x, x) @ Y) / (x @ x)
+                    val += lam / (p - 1) * max(1.0 - v, 0.0) ** (1 / a)
+    return val
+
+
+def test_beta_one_half_is_the_papers_data_term_and_beta_only_rescales_lambda():
+    G = noisy_mean(9, 30, 60, sigma=0.5, outliers=2, scale_spread=True)
+    base = fo.fa_aggregate(G, 3, 0.2, iters=6)
+    same = fo.fa_aggregate(G, 3, 0.2, iters=6, alpha=1.0, beta=0.5)
+    assert np.array_equal(base["d"], same["d"]) and base["objective"] == same["objective"]
+    # alpha = 1: the data term is 2(1-beta) times the paper's, i.e. the paper's problem with lambda / (2(1-beta))
+    # (from a common start: the uniform first round does not know about beta)
+    b = 0.8
+    Y0 = rng(66).standard_normal((30, 3))
+    other = fo.fa_aggregate(G, 3, 0.2, iters=6, beta=b, method="qr", Y0=Y0)
+    scaled = fo.fa_aggregate(G, 3, 0.2 / (2 * (1 - b)), iters=6, Y0=Y0)
+    assert fo.principal_angles(other["Y"], scaled["Y"]).max() < 1e-8
+    assert np.allclose(np.asarray(other["objective"]) / (2 * (1 - b)), scaled["objective"], rtol=1e-9)
+    # without the regulariser beta does not matter at all
+    assert fo.principal_angles(fo.fa_aggregate(G, 3, 0.0, iters=6, beta=0.9)["Y"],
+                               fo.fa_aggregate(G, 3, 0.0, iters=6)["Y"]).max() < 1e-8
+
+
+def test_indefinite_weighted_pca_by_qr_matches_the_n_by_n_matrix():
+    r = rng(61)
+    G = r.standard_normal((6, 9))
+    w = r.standard_normal(6)                       # both signs
+    W = np.abs(r.standard_normal((6, 6))) * 0.1
+    W = W + W.T
+    np.fill_diagonal(W, 0.0)
+    Yq, eq = fo.weighted_pca_qr(G, w, W, 3)
+    Yl, el = fo.weighted_pca_literal(G, w, W, 3)
+    assert Yq.shape == Yl.shape and fo.principal_angles(Yq, Yl).max() < 1e-9
+    assert np.allclose(np.sort(eq)[::-1][:3], np.sort(el)[::-1][:3], rtol=1e-10)
+    # all weights negative: nothing has a positive eigenvalue, Y is empty
+    Yn, _ = fo.weighted_pca_qr(G, -np.abs(w), 0 * W, 3)
+    assert Yn.shape[1] == 0
+
+
+@pytest.mark.parametrize("alpha,beta,lam,a", [(0.7, 0.5, 0.0, 2.0), (0.5, 0.3, 0.3, 2.0), (0.8, 0.5, 0.2, 3.0)])
+def test_beta_likelihood_descends_and_reaches_a_local_minimum(alpha, beta, lam, a):
+    n, p, m = 12, 10, 3
+    G = noisy_mean(p, n, 62, sigma=0.6, outliers=2, scale_spread=True)
+    out = fo.fa_aggregate(G, m, lam, iters=400, a=a, alpha=alpha, beta=beta)
+    objs = out["objective"]
+    assert all(objs[t + 1] <= objs[t] + 1e-10 for t in range(len(objs) - 1))
+    Y = out["Y"]
+    assert abs(objs[-1] - beta_objective(G, Y, lam, a, alpha, beta)) < 1e-7
+    if Y.shape[1] == m:
+        base = beta_objective(G, Y, lam, a, alpha, beta)
+        r = rng(63)
+        worst = 0.0
+        for _ in range(60):
+            D = r.standard_normal((n, m))
+            D -= Y @ (Y.T @ D)
+            D /= np.linalg.norm(D)
+            for t in (1e-2, 1e-3, 1e-4):
+                Q, _ = np.linalg.qr(Y + t * D)
+                worst = max(worst, (base - beta_objective(G, Q, lam, a, alpha, beta)) / t)
+        assert worst < 1e-5
+
+
+def test_beta_likelihood_brute_force_in_the_plane():
+    G = _clustered(2, 7, 64, outliers=2)
+    alpha, beta, lam = 0.6, 0.5, 0.2
+    out = fo.fa_aggregate(G, 1, lam, iters=300, alpha=alpha, beta=beta)
+    k = 6000
+    grid = _line_grid_2d(k)
+    vals = np.asarray([beta_objective(G, y[:, None], lam, 2.0, alpha, beta) for y in grid])
+    is_min = (vals <= np.roll(vals, 1)) & (vals <= np.roll(vals, -1))
+    assert out["Y"].shape[1] == 1
+    # each term moves by at most the angle step times its coefficient (roots of values in [0, 1])
+    resolution = (np.pi / k) * (7 * (2 * (1 - beta) + 2 * (1 - alpha)) + 2 * lam * 7) * 40
+    assert np.min(np.abs(vals[is_min] - out["objective"][-1])) < resolution
+
+
+def test_beta_arguments():
+    G = noisy_mean(5, 8, 65)
+    for bad in (dict(alpha=0.0), dict(alpha=1.5), dict(beta=0.0), dict(beta=1.2)):
+        with pytest.raises(ValueError):
+            fo.fa_aggregate(G, 2, **bad)
