@@ -121,6 +121,22 @@ int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double 
                     int iters, float* out, double* A_out, double* S_out, void* ws, size_t ws_bytes,
                     int* status, void* stream);
 
+/* General Beta(alpha, beta) likelihood of the values v_i (Eq. (1) has alpha = 1, beta = 1/2; the
+ * extension paragraph of Section 2.2 allows any shape parameters, "two terms" in the surrogate).
+ * With the surrogate of Eq. (4) on both logarithms the data term of worker i becomes
+ *     2 (1 - beta) (1 - v_i)^(1/a) + 2 (1 - alpha) v_i^(1/a)
+ * (alpha = 1, beta = 1/2: the term of Eq. (5)); the regulariser is unchanged.  Both parts are concave
+ * in v_i for 0 < alpha <= 1, 0 < beta <= 1 -- other values are an argument error -- so each round is
+ * still one weighted eigenproblem; weights can be negative and only directions with a positive
+ * eigenvalue enter Y (FA_ST_RANK_LT_M reports fewer than m). */
+int fa_irls_beta(const double* K, int p, int m, double lambda, double a, double alpha, double beta,
+                 int iters, double* A_out, float* c_out, double* w_out, double* obj_out,
+                 int* status, void* stream);
+
+int fa_aggregate_beta(const void* G, int dtype, int p, long long n, int m, double lambda, double a,
+                      double alpha, double beta, int iters, float* out, double* A_out, void* ws,
+                      size_t ws_bytes, int* status, void* stream);
+
 /* IRLS that starts from a given subspace and may stop early.
  *   A0   : p x m fp64 row-major or NULL.  The first reweighting uses the term values at span(G^T A0)
  *          instead of uniform weights (the "smart initialization" Section 2.1 mentions): pass the

@@ -38,13 +38,15 @@ _lib.fa_irls_multi.argtypes = [_vp, _i, _vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, 
 _lib.fa_aggregate_multi.argtypes = [_vp, _i, _i, _ll, _vp, _i, _i, _d, _d, _i, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_irls_warm.argtypes = [_vp, _i, _i, _d, _d, _i, _d, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.fa_aggregate_warm.argtypes = [_vp, _i, _i, _ll, _i, _d, _d, _i, _d, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.fa_irls_beta.argtypes = [_vp, _i, _i, _d, _d, _d, _d, _i, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.fa_aggregate_beta.argtypes = [_vp, _i, _i, _ll, _i, _d, _d, _d, _d, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_combine.argtypes = [_vp, _i, _i, _ll, _vp, _vp, _vp]
 _lib.fa_aggregate.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_aggregate_host.argtypes = [_vp, _i, _i, _ll, _i, _d, _i, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.fa_gram_static.argtypes = [_vp, _i, _i, _ll, _vp, _vp]
 _lib.fa_gram_static.restype = _i
 for _name in ("fa_workspace_bytes", "fa_gram", "fa_irls_step", "fa_irls", "fa_irls_ex", "fa_aggregate_ex",
-              "fa_irls_multi", "fa_aggregate_multi", "fa_irls_warm", "fa_aggregate_warm", "fa_combine", "fa_aggregate", "fa_aggregate_host"):
+              "fa_irls_multi", "fa_aggregate_multi", "fa_irls_warm", "fa_aggregate_warm", "fa_irls_beta", "fa_aggregate_beta", "fa_combine", "fa_aggregate", "fa_aggregate_host"):
     getattr(_lib, _name).restype = _i
 
 
@@ -191,6 +193,28 @@ def fa_aggregate_warm(G, m, lam, iters, a=2.0, tol=-1.0, A0=None, out=None, A_ou
                                   _dev(out, torch.float32, n, "out"), _ptr(A_out), _ptr(rounds_out), ws.data_ptr(),
                                   ws.numel() * ws.element_size(), _ptr(status), _stream(stream)),
            "fa_aggregate_warm")
+    return out
+
+
+def fa_irls_beta(K, m, lam, iters, alpha, beta, a=2.0, A_out=None, c_out=None, w_out=None, obj_out=None, status=None,
+                 stream=None):
+    """IRLS with a Beta(alpha, beta) likelihood of the workers' values (alpha = 1, beta = 1/2: fa_irls)."""
+    p = int(K.shape[0])
+    c_out = torch.empty(p, dtype=torch.float32, device=K.device) if c_out is None else c_out
+    _check(_lib.fa_irls_beta(_dev(K, torch.float64, p * p, "K"), p, m, float(lam), float(a), float(alpha), float(beta),
+                             iters, _ptr(A_out), _dev(c_out, torch.float32, p, "c_out"), _ptr(w_out), _ptr(obj_out),
+                             _ptr(status), _stream(stream)), "fa_irls_beta")
+    return c_out
+
+
+def fa_aggregate_beta(G, m, lam, iters, alpha, beta, a=2.0, out=None, A_out=None, ws=None, status=None, stream=None):
+    code, p, n = _gradients(G)
+    out = torch.empty(n, dtype=torch.float32, device=G.device) if out is None else out
+    ws = new_workspace(G, m) if ws is None else ws
+    _check(_lib.fa_aggregate_beta(G.data_ptr(), code, p, n, m, float(lam), float(a), float(alpha), float(beta), iters,
+                                  _dev(out, torch.float32, n, "out"), _ptr(A_out), ws.data_ptr(),
+                                  ws.numel() * ws.element_size(), _ptr(status), _stream(stream)),
+           "fa_aggregate_beta")
     return out
 
 

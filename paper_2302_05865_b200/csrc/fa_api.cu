@@ -107,6 +107,7 @@ int fa_irls_step(const double* K, int p, int m, double lambda, int first, double
       (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
   fa::IrlsArgs a{};
+  a.cb = 1.0; a.ca = 0.0;
   a.K = K; a.p = p; a.m = m; a.iters = 1; a.lambda = lambda; a.a = 2.0; a.start_from_A = first ? 0 : 1;
   a.A0 = A; a.tol = -1.0;
   a.A = A; a.w = w; a.obj = objective; a.status = status;
@@ -115,7 +116,8 @@ int fa_irls_step(const double* K, int p, int m, double lambda, int first, double
 
 static int irls_common(const double* K, int p, int m, double lambda, double a, int iters, double tol, const double* A0,
                        double* A_out, float* c_out, double* S_out, double* w_out, double* obj_out, int* rounds_out,
-                       int* status, void* stream) {
+                       int* status, void* stream, double alpha = 1.0, double beta = 0.5) {
+  if (!(alpha > 0.0 && alpha <= 1.0 && beta > 0.0 && beta <= 1.0)) return FA_ERR_ARG;
   if (!K || !c_out || p < 1 || p > FA_MAX_P || m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda) ||
       !(a > 1.0) || isinf(a) || isnan(tol))
     return FA_ERR_ARG;
@@ -125,8 +127,10 @@ static int irls_common(const double* K, int p, int m, double lambda, double a, i
       (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
   fa::IrlsArgs args{};
+  args.cb = 1.0; args.ca = 0.0;
   args.K = K; args.p = p; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a;
   args.start_from_A = A0 ? 2 : 0; args.A0 = A0; args.tol = tol; args.rounds = rounds_out;
+  if (!(alpha == 1.0 && beta == 0.5)) { args.cb = 2.0 * (1.0 - beta); args.ca = 2.0 * (1.0 - alpha); }
   args.A = A_out; args.c = c_out; args.S = S_out; args.w = w_out; args.obj = obj_out; args.status = status;
   return fa::launch_irls(args, static_cast<cudaStream_t>(stream)) == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
@@ -135,6 +139,12 @@ int fa_irls_ex(const double* K, int p, int m, double lambda, double a, int iters
                double* S_out, double* w_out, double* obj_out, int* status, void* stream) {
   return irls_common(K, p, m, lambda, a, iters, -1.0, nullptr, A_out, c_out, S_out, w_out, obj_out, nullptr, status,
                      stream);
+}
+
+int fa_irls_beta(const double* K, int p, int m, double lambda, double a, double alpha, double beta, int iters,
+                 double* A_out, float* c_out, double* w_out, double* obj_out, int* status, void* stream) {
+  return irls_common(K, p, m, lambda, a, iters, -1.0, nullptr, A_out, c_out, nullptr, w_out, obj_out, nullptr, status,
+                     stream, alpha, beta);
 }
 
 int fa_irls_warm(const double* K, int p, int m, double lambda, double a, int iters, double tol, const double* A0,
@@ -170,6 +180,7 @@ int fa_aggregate_ex(const void* G, int dtype, int p, long long n, int m, double 
   if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
   if (fa::launch_gram(G, dtype, p, n, w.partials, w.counter, w.Kbuf, status, st) != cudaSuccess) return FA_ERR_CUDA;
   fa::IrlsArgs args{};
+  args.cb = 1.0; args.ca = 0.0;
   args.K = w.Kbuf;
   args.p = p; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a; args.start_from_A = 0;
   args.tol = -1.0;
@@ -190,6 +201,7 @@ int fa_irls_multi(const double* K, int rows, const int* counts, int workers, int
       (status && !fa::aligned(status, 4)))
     return FA_ERR_ALIGN;
   fa::IrlsArgs args{};
+  args.cb = 1.0; args.ca = 0.0;
   args.K = K; args.p = rows; args.m = m; args.iters = iters; args.lambda = lambda; args.a = a; args.start_from_A = 0;
   args.tol = -1.0;
   args.A = A_out; args.c = c_out; args.S = S_out; args.w = w_out; args.obj = obj_out; args.status = status;
@@ -216,6 +228,28 @@ int fa_aggregate_multi(const void* G, int dtype, int rows, long long n, const in
                          stream);
   if (rc != FA_OK) return rc;
   if (fa::launch_combine(G, dtype, rows, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
+  return FA_OK;
+}
+
+int fa_aggregate_beta(const void* G, int dtype, int p, long long n, int m, double lambda, double a, double alpha,
+                      double beta, int iters, float* out, double* A_out, void* ws, size_t ws_bytes, int* status,
+                      void* stream) {
+  if (!G || !out || !ws || !fa::shape_ok(p, n, dtype)) return FA_ERR_ARG;
+  if (m < 1 || m > p || iters < 1 || !(lambda >= 0.0) || isinf(lambda) || !(a > 1.0) || isinf(a) ||
+      !(alpha > 0.0 && alpha <= 1.0 && beta > 0.0 && beta <= 1.0))
+    return FA_ERR_ARG;
+  if (!fa::aligned(G, dtype == FA_F32 ? 4 : 2) || !fa::aligned(out, 4) || !fa::aligned(ws, 16) ||
+      (A_out && !fa::aligned(A_out, 8)) || (status && !fa::aligned(status, 4)))
+    return FA_ERR_ALIGN;
+  fa::Workspace w = fa::carve_ws(ws, p, n, dtype);
+  if (ws_bytes < w.total) return FA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (status && cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return FA_ERR_CUDA;
+  if (fa::launch_gram(G, dtype, p, n, w.partials, w.counter, w.Kbuf, status, st) != cudaSuccess) return FA_ERR_CUDA;
+  int rc = irls_common(w.Kbuf, p, m, lambda, a, iters, -1.0, nullptr, A_out, w.c, nullptr, nullptr, nullptr, nullptr,
+                       status, stream, alpha, beta);
+  if (rc != FA_OK) return rc;
+  if (fa::launch_combine(G, dtype, p, n, w.c, out, st) != cudaSuccess) return FA_ERR_CUDA;
   return FA_OK;
 }
 

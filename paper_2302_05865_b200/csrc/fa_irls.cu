@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   fa_irls::carve(s, irls_smem, a.p, ctx.nt);
   fa_irls::Outputs o{a.A, a.c, a.w, a.obj, a.S, a.status, a.rounds};
   const int st = fa_irls::run<(NT > 192)>(ctx, s, K, a.p, a.m, a.lambda, a.a, a.iters, a.start_from_A, a.A0, a.tol, o,
-                                           a.workers, a.counts);
+                                           a.workers, a.counts, a.cb, a.ca);
   if (st && a.status && ctx.tid == 0) atomicOr(a.status, st);
 }
 

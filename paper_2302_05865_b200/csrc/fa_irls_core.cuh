@@ -373,8 +373,12 @@ FA_FN void term_of(double u, double a, double& contrib, double& denom) {
 // From residual coordinates Res (rows k0..r-1 are the part of f_i outside the subspace) and the
 // full coordinates P: u_i, next data weights w_i, the matrix M of the next weighted PCA and the
 // value of Eq. (5).  `uniform` builds the round-one weights instead (u is not needed then).
+//
+// cb, ca: the data term of worker i is cb (1 - v_i)^(1/a) + ca v_i^(1/a) -- a Beta(alpha, beta)
+// likelihood of the values with cb = 2 (1 - beta), ca = 2 (1 - alpha); Eq. (1) has alpha = 1,
+// beta = 1/2, i.e. cb = 1, ca = 0.  With ca > 0 a weight can be negative.
 FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
-                                   double coef, bool uniform, double a) {
+                                   double coef, bool uniform, double a, double cb = 1.0, double ca = 0.0) {
   const int ld = s.ld;
   double part = 0.0;
   for (int i = c.tid; i < p; i += c.nt) {
@@ -387,8 +391,24 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
         ui = acc / s.fn[i];
         double contrib, denom;
         term_of(ui, a, contrib, denom);
-        part += contrib;
-        wi = 1.0 / (s.fn[i] * denom);
+        if (cb == 1.0 && ca == 0.0) {
+          part += contrib;
+          wi = 1.0 / (s.fn[i] * denom);
+        } else {
+          // explained part: the leading coordinates when Res is the coordinate matrix itself
+          double vi;
+          if (Res == s.P) {
+            double e = 0.0;
+            for (int k = 0; k < k0; ++k) { double v = s.P[k * ld + i]; e += v * v; }
+            vi = e / s.fn[i];
+          } else {
+            vi = fmax(1.0 - ui, 0.0);
+          }
+          double contrib_v, denom_v;
+          term_of(vi, a, contrib_v, denom_v);
+          part += cb * contrib + ca * contrib_v;
+          wi = (cb / denom - ca / denom_v) / s.fn[i];
+        }
       }
     }
     s.u[i] = ui;
@@ -537,7 +557,7 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
 template <bool LARGE>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
               int start, const double* A0, double tol, const Outputs& o, int nw = 0,
-              const unsigned char* cnt = nullptr) {
+              const unsigned char* cnt = nullptr, double cb = 1.0, double ca = 0.0) {
   const int ld = s.ld;
   const int pp = (p + 1) & ~1;
   int status = 0;
@@ -725,7 +745,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   }
   if (start == 0) {
     if (grouped) (void)weights_and_objective_grouped(c, s, s.P, 0, r, p, coef, true, a);
-    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a);
+    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a, cb, ca);
   } else {
     // C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
     for (int idx = c.tid; idx < m * p; idx += c.nt) {
@@ -743,7 +763,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
     c.sync();
     if (grouped) (void)weights_and_objective_grouped(c, s, s.tmp, 0, r, p, coef, false, a);
-    else (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a);
+    else (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a, cb, ca);
   }
 
   int m_eff = 0, rounds = iters;
@@ -807,7 +827,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
 
     // ---- terms of Eq. (5) at the new subspace, and the next round's weights
     double obj = grouped ? weights_and_objective_grouped(c, s, s.P, m_eff, r, p, coef, false, a)
-                         : weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a);
+                         : weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a, cb, ca);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
     if (tol >= 0.0 && t >= 1 && fabs(prev_obj - obj) <= tol) {      // same value in every thread
       rounds = t + 1;

@@ -25,6 +25,7 @@ struct IrlsArgs {
   int p, m, iters;
   double lambda;
   double a;          // surrogate constant of Eq. (4); 2 = the paper's square roots
+  double cb, ca;     // data term cb (1-v)^(1/a) + ca v^(1/a): 2(1-beta), 2(1-alpha) of a Beta likelihood; 1, 0 = Eq. (1)
   int start_from_A;  // 0 uniform first round; 1 start from A0 (orthonormal image); 2 start from any A0
   const double* A0;  // p x m, read before A is written (may alias A)
   double tol;        // >= 0: stop once the objective moved by <= tol; < 0: run all rounds

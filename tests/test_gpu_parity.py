@@ -438,3 +438,47 @@ def test_aggregate_continues_from_the_previous_steps_subspace(fa):
     assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < 1e-4
     with pytest.raises(fa.FaError):
         fa.fa_aggregate_warm(G2, m, lam, 5, tol=float("nan"))
+
+
+BETA_CASES = [
+    (15, 2000, "noisy_mean", 8, 0.01, 2.0, 0.7, 0.5, 8), (7, 33, "dup_zero", 3, 0.2, 2.0, 0.5, 0.3, 6),
+    (31, 3000, "noisy_mean", 12, 0.01, 3.0, 0.8, 0.5, 8), (64, 300, "noisy_mean", 20, 0.01, 2.0, 0.9, 0.6, 6),
+    (15, 2000, "gauss", 8, 0.1, 2.0, 1.0, 0.8, 6),
+    # weights of both signs, and all negative (nothing enters Y)
+    (12, 400, "gauss", 6, 0.5, 2.0, 0.3, 0.8, 6), (15, 2000, "noisy_mean", 8, 0.5, 2.0, 0.4, 0.8, 6),
+    (9, 100, "noisy_mean", 4, 1.0, 2.0, 0.5, 0.9, 6), (10, 50, "noisy_mean", 5, 0.0, 2.0, 0.3, 0.9, 6),
+]
+
+
+@pytest.mark.parametrize("p,n,kind,m,lam,a,alpha,beta,iters", BETA_CASES)
+def test_irls_with_a_general_beta_likelihood(fa, p, n, kind, m, lam, a, alpha, beta, iters):
+    G = si.ladder_case(p, n, 9, kind).astype(np.float64)
+    ref = fo.fa_aggregate(G, m, lam, iters, a=a, alpha=alpha, beta=beta)
+    K = torch.from_numpy(fo.inner_products(G)).cuda()
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    w = torch.zeros(p, dtype=torch.float64, device="cuda")
+    obj = torch.zeros(iters, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    c = fa.fa_irls_beta(K, m, lam, iters, alpha, beta, a=a, A_out=A, w_out=w, obj_out=obj, status=status)
+    torch.cuda.synchronize()
+    k = ref["Y"].shape[1]
+    st = int(status.item())
+    assert st & ~fa.ST_RANK_LT_M == 0 and bool(st & fa.ST_RANK_LT_M) == (k < m)
+    if k:
+        assert fo.principal_angles(ref["Y"], G.T @ A.cpu().numpy()[:, :k]).max() < 1e-7
+    assert not A.cpu().numpy()[:, k:].any()
+    assert np.allclose(obj.cpu().numpy(), ref["objective"], rtol=1e-9, atol=1e-9)
+    assert np.allclose(w.cpu().numpy(), ref["w"], rtol=1e-6, atol=1e-12 * np.abs(ref["w"]).max())
+    assert fo.rel_l2(c.cpu().numpy().astype(np.float64) @ G, ref["d"]) < 1e-6 or not ref["d"].any()
+
+
+def test_aggregate_with_a_general_beta_likelihood(fa):
+    G_np = si.ladder_case(15, 90_001, 4, "noisy_mean")
+    G = torch.from_numpy(G_np).cuda()
+    out = fa.fa_aggregate_beta(G, 8, 0.05, 7, 0.6, 0.7)
+    ref = fo.fa_aggregate(G_np.astype(np.float64), 8, 0.05, 7, alpha=0.6, beta=0.7)
+    assert fo.rel_l2(out.cpu().numpy(), ref["d"]) < 1e-4
+    assert torch.equal(fa.fa_aggregate_beta(G, 8, 0.05, 7, 1.0, 0.5), fa.fa_aggregate(G, 8, 0.05, 7))
+    for alpha, beta in ((0.0, 0.5), (1.5, 0.5), (1.0, 0.0), (1.0, 1.5), (float("nan"), 0.5)):
+        with pytest.raises(fa.FaError):
+            fa.fa_aggregate_beta(G, 8, 0.05, 7, alpha, beta)
