@@ -40,9 +40,17 @@ __device__ __forceinline__ double fa_fast_rsqrt(double x) {
   y = y * fma(-hx * y, y, 1.5);
   return y;
 }
+// The bare hardware approximation (relative error about 2^-22).
+__device__ __forceinline__ double fa_approx_rsqrt(double x) {
+  double y;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  return y;
+}
 #define FA_RSQRT(x) fa_fast_rsqrt(x)
+#define FA_RSQRT_APPROX(x) fa_approx_rsqrt(x)
 #else
 #define FA_RSQRT(x) (1.0 / sqrt(x))
+#define FA_RSQRT_APPROX(x) (1.0 / sqrt(x))
 #endif
 
 namespace fa_irls {
@@ -129,58 +137,112 @@ FA_FN double block_sum(const Ctx& c, const Smem& s, double v) {
 #endif
 }
 
-// Round-robin pairing: in round rd of a sweep over pp (even) indices, pair k is (a, b), a < b.
-FA_FN void pair_of(int rd, int k, int pp, int& a, int& b) {
-  if (k == 0) { a = pp - 1; b = rd; }
-  else {
-    a = rd + k; if (a >= pp - 1) a -= pp - 1;
-    b = rd + (pp - 1) - k; if (b >= pp - 1) b -= pp - 1;
-  }
-  if (a > b) { int t = a; a = b; b = t; }
-}
-
-// Rotation (cs, sn) that annihilates T[a][b]; identity for padded indices and for entries at
-// rounding level.  Written from the double angle, without division and with two rsqrt:
+// Rotation (cs, sn) for a pair with diagonal entries app, aqq and off-diagonal entry apq; identity
+// for entries at rounding level.  From the double angle, without division:
 //   d = a_qq - a_pp, h = 2 a_pq, cos 2phi = |d| / sqrt(d^2 + h^2),
 //   c = sqrt((1 + cos 2phi) / 2), s = sign(d) * h / (2 c sqrt(d^2 + h^2)).
+// The reciprocal square roots start from the hardware approximation (22 bits).  The first gets one
+// Newton step (44 bits): it alone fixes the angle, s / c = hr / x, and an angle that is off by
+// 1e-13 relative leaves 1e-13 of the entry it was meant to annihilate.  The second only scales c
+// and s together, and a Jacobi rotation has to be ORTHOGONAL to full accuracy for the similarity
+// transform to be exact; so (c, s) is scaled onto the unit circle at the end:
+// c^2 + s^2 = 1 + e with |e| ~ 1e-6, factor 1 - e/2 + 3 e^2 / 8, error e^3.  This keeps the chain of
+// dependent fp64 operations (8 cycles each, the unit of cost in this kernel) short; there is no
+// branch, so two rotations worked out by one thread overlap.
 // Returns true when the entry was "large" (above kJacobiBig relative to its diagonal).
-FA_FN bool rotation(const double* T, int ld, int a, int b, int dim, double& cs, double& sn) {
-  cs = 1.0; sn = 0.0;
-  if (b >= dim) return false;
-  const double app = T[a * ld + a], aqq = T[b * ld + b], apq = T[a * ld + b];
+FA_FN bool rotation_of(double app, double aqq, double apq, double& cs, double& sn) {
   const double m2 = apq * apq, ref2 = fabs(app * aqq);
-  if (!(m2 > (kJacobiTol * kJacobiTol) * ref2 && m2 > 1e-280)) return false;
+  const bool ok = (m2 > (kJacobiTol * kJacobiTol) * ref2) && (m2 > 1e-280);
   const double d = aqq - app, h = 2.0 * apq;
-  const double rinv = FA_RSQRT(d * d + h * h);
-  const double x = 0.5 + 0.5 * fabs(d) * rinv;          // cos^2 phi, in [1/2, 1]
-  const double cinv = FA_RSQRT(x);
-  cs = x * cinv;
-  sn = 0.5 * h * rinv * cinv;
-  if (d < 0.0) sn = -sn;
-  return m2 > (kJacobiBig * kJacobiBig) * ref2;
+  const double q = fma(d, d, h * h);
+  const double qs = ok ? q : 1.0;
+  double rinv = FA_RSQRT_APPROX(qs);
+  rinv = rinv * fma((-0.5 * qs) * rinv, rinv, 1.5);      // one Newton step: the angle (s / c = hr / x) depends on rinv only
+  const double hr = (0.5 * h) * rinv;
+  const double x = fma(0.5 * fabs(d), rinv, 0.5);        // cos^2 phi, in [1/2, 1]
+  const double cinv = FA_RSQRT_APPROX(x);
+  double c = x * cinv, sv = hr * cinv;
+  const double e = fma(c, c, fma(sv, sv, -1.0));
+  const double f = fma(e, fma(e, 0.375, -0.5), 1.0);
+  c *= f;
+  sv *= f;
+  cs = ok ? c : 1.0;
+  sn = ok ? (d < 0.0 ? -sv : sv) : 0.0;
+  return ok && (m2 > (kJacobiBig * kJacobiBig) * ref2);
 }
 
-// Cyclic Jacobi with round-robin pairing.  T (dim x dim, symmetric, both halves stored, rows and
-// columns dim..pp-1 zero) is driven to diagonal form; J accumulates the rotations (J <- J * R).
-// One barrier per round: every work item recomputes the one or two rotations it needs from the
-// round's input matrix (double-buffered in T / Talt), so no thread waits for another thread's
-// parameters.  A pair is rotated whenever its off-diagonal entry is above rounding level;
-// sweeping stops after the first sweep in which no rotated entry exceeded kJacobiBig relative to
-// its diagonal: that sweep's rotations leave entries of the order of its square (quadratic
-// convergence of the cyclic method), i.e. below rounding level.
-// On return *Tio points at the buffer that holds the diagonalised matrix.  Returns the sweeps made.
-template <bool LARGE>
-FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double* J, int dim, int jrows) {
+FA_FN bool rotation(const double* T, int ld, int a, int b, int dim, double& cs, double& sn) {
+  if (b >= dim) { cs = 1.0; sn = 0.0; return false; }
+  return rotation_of(T[a * ld + a], T[b * ld + b], T[a * ld + b], cs, sn);
+}
+
+// Systolic (Brent-Luk) arrangement of np pairs: pair k sits at positions (k, np + k) -- "top" entries
+// in the first half, "bottom" entries in the second, so that threads with consecutive pair numbers
+// touch consecutive shared-memory words.  After a round top_0 stays, the other top entries move one
+// pair up, the bottom entries one pair down, and the two ends cross over (bottom_0 -> top_1,
+// top_{np-1} -> bottom_{np-1}).  pp - 1 rounds pair every two indices exactly once and bring every
+// index back to where it started.  Returns where the content of position x goes.
+FA_FN int systolic_next(int x, int np) {
+  if (x == 0) return 0;
+  if (x < np) return x == np - 1 ? 2 * np - 1 : x + 1;      // top_k, k >= 1
+  return x == np ? (np > 1 ? 1 : np) : x - 1;                // bottom_k
+}
+
+// Cyclic Jacobi, all pairs of a round in parallel.  T (dim x dim, symmetric, both halves stored, rows
+// and columns dim..pp-1 zero) is driven to diagonal form; J accumulates the rotations (J <- J * R).
+// A pair is rotated whenever its off-diagonal entry is above rounding level; sweeping stops after
+// the first sweep in which no rotated entry exceeded kJacobiBig relative to its diagonal: that
+// sweep's rotations leave entries of the order of its square (quadratic convergence of the cyclic
+// method), i.e. below rounding level.
+//
+// The data MOVES instead of the pairing (Brent-Luk systolic arrangement): a round rotates the pairs
+// at the fixed positions (k, np + k) and stores rows and columns (and the columns of J) at their
+// systolic_next() positions, from T / J into Talt / Jalt and back.  So every thread owns the same
+// 2x2 blocks of T and (row, pair) items of J for the whole solve, all its offsets are worked out
+// once before the first sweep, and all its loads go out together at the top of a round -- what a
+// round costs here is the number of dependent instructions a warp has to issue.
+//   * up to 8 pairs (dim <= 16): one item per thread; each thread works out the one or two
+//     rotations it needs itself: one barrier per round and nothing else between threads;
+//   * more pairs: several items per thread; the rotations are worked out once by the first np
+//     threads and published in shared memory (a second barrier per round).
+// A full sweep (pp - 1 rounds) returns every index to its own position, and sweeps are never cut
+// short.  On return *Tio / *Jio point at the buffers that hold the results.  Returns the sweeps made.
+// Up to 8 pairs on the device; any size on the host.
+FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
+                       int dim, int jrows) {
   const int ld = s.ld;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
-  if (dim < 2) return 0;
   double* T = *Tio;
   double* Tn = *Taltio;
-  int sh = 0;
-  while ((1 << sh) < np) ++sh;             // items are indexed (k, l) = (idx >> sh, idx & mask)
-  const int mask = (1 << sh) - 1;
-  const int nblk = np << sh, nrow = jrows << sh;
+  double* J = *Jio;
+  double* Jn = *Jaltio;
+  const int nb2 = np * np, total2 = nb2 + jrows * np;
+  // the item this thread owns for the whole solve (element offsets into T / J)
+  struct Item { int kind, diag, kaa, kbb, kab, laa, lbb, lab, x0, x1, x2, x3, z0, z1, z2, z3; } it;
+  it.kind = 0;
+  {
+    const int idx = c.tid;
+    if (idx < nb2) {
+      const int k = idx / np, l = idx - k * np;
+      const int a = k, b = np + k, cc = l, d = np + l;
+      const int pa = systolic_next(a, np), pb = systolic_next(b, np), pc = systolic_next(cc, np), pd = systolic_next(d, np);
+      it.kind = 1; it.diag = (k == l);
+      it.kaa = a * ld + a; it.kbb = b * ld + b; it.kab = a * ld + b;
+      it.laa = cc * ld + cc; it.lbb = d * ld + d; it.lab = cc * ld + d;
+      it.x0 = a * ld + cc; it.x1 = a * ld + d; it.x2 = b * ld + cc; it.x3 = b * ld + d;
+      it.z0 = pa * ld + pc; it.z1 = pa * ld + pd; it.z2 = pb * ld + pc; it.z3 = pb * ld + pd;
+    } else if (idx < total2) {
+      const int q = idx - nb2;
+      const int x = q / np, l = q - x * np;
+      const int cc = l, d = np + l;
+      it.kind = 2; it.diag = 0;
+      it.laa = cc * ld + cc; it.lbb = d * ld + d; it.lab = cc * ld + d;
+      it.x0 = x * ld + cc; it.x1 = x * ld + d;
+      it.z0 = x * ld + systolic_next(cc, np); it.z1 = x * ld + systolic_next(d, np);
+      it.kaa = it.kbb = it.kab = it.x2 = it.x3 = it.z2 = it.z3 = 0;
+    }
+  }
   int sweep = 0;
   // "large rotation in this sweep" flag, double-buffered by sweep parity (slots 0 and 3)
   if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
@@ -189,151 +251,202 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
     int* big = &s.flags[(sweep & 1) ? 3 : 0];
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
-#ifndef FA_IRLS_HOST
-      if (LARGE && np > 8) {
-        // Larger problems: the np rotations are computed once, by the first np threads, and published
-        // in shared memory (one extra barrier); redundant fp64 work would otherwise fill the pipe.
-        // Items are then taken three at a time, all loads first, so their latencies overlap.
-        if (c.tid < np) {
-          int a, b;
-          double cs, sn;
-          pair_of(rd, c.tid, pp, a, b);
-          if (rotation(T, ld, a, b, dim, cs, sn)) *big = 1;
-          s.ra[c.tid] = a; s.rb[c.tid] = b; s.rc[c.tid] = cs; s.rs[c.tid] = sn;
-        }
-        c.sync();
-        const int total = nblk + nrow;
-#ifndef FA_IRLS_BATCH
-#define FA_IRLS_BATCH 2
-#endif
-        constexpr int U = FA_IRLS_BATCH;
-        for (int base = c.tid; base < total; base += U * c.nt) {
-          int kind[U], ia[U], ib[U], ic[U], id[U];
-          double rk_c[U], rk_s[U], rl_c[U], rl_s[U], x0[U], x1[U], x2[U], x3[U];
-#pragma unroll
-          for (int u = 0; u < U; ++u) {
-            const int idx = base + u * c.nt;
-            kind[u] = 0;
-            if (idx < nblk) {
-              const int k = idx >> sh, l = idx & mask;
-              if (l < np) {
-                kind[u] = 1;
-                ia[u] = s.ra[k]; ib[u] = s.rb[k]; ic[u] = s.ra[l]; id[u] = s.rb[l];
-                rk_c[u] = s.rc[k]; rk_s[u] = s.rs[k]; rl_c[u] = s.rc[l]; rl_s[u] = s.rs[l];
-                x0[u] = T[ia[u] * ld + ic[u]]; x1[u] = T[ia[u] * ld + id[u]];
-                x2[u] = T[ib[u] * ld + ic[u]]; x3[u] = T[ib[u] * ld + id[u]];
-                if (k == l && rk_s[u] != 0.0) kind[u] = 3;   // diagonal block: the rotated entry is exactly zero
-              }
-            } else if (idx < total) {
-              const int q = idx - nblk;
-              const int x = q >> sh, k = q & mask;
-              if (k < np && s.rs[k] != 0.0) {
-                kind[u] = 2;
-                ia[u] = x * ld + s.ra[k]; ib[u] = x * ld + s.rb[k];
-                rk_c[u] = s.rc[k]; rk_s[u] = s.rs[k];
-                x0[u] = J[ia[u]]; x1[u] = J[ib[u]];
-              }
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < U; ++u) {
-            if (kind[u] == 1 || kind[u] == 3) {
-              const double yac = rk_c[u] * x0[u] - rk_s[u] * x2[u], yad = rk_c[u] * x1[u] - rk_s[u] * x3[u];
-              const double ybc = rk_s[u] * x0[u] + rk_c[u] * x2[u], ybd = rk_s[u] * x1[u] + rk_c[u] * x3[u];
-              double zac = rl_c[u] * yac - rl_s[u] * yad, zad = rl_s[u] * yac + rl_c[u] * yad;
-              double zbc = rl_c[u] * ybc - rl_s[u] * ybd, zbd = rl_s[u] * ybc + rl_c[u] * ybd;
-              if (kind[u] == 3) { zad = 0.0; zbc = 0.0; }
-              Tn[ia[u] * ld + ic[u]] = zac; Tn[ia[u] * ld + id[u]] = zad;
-              Tn[ib[u] * ld + ic[u]] = zbc; Tn[ib[u] * ld + id[u]] = zbd;
-            } else if (kind[u] == 2) {
-              J[ia[u]] = rk_c[u] * x0[u] - rk_s[u] * x1[u];
-              J[ib[u]] = rk_s[u] * x0[u] + rk_c[u] * x1[u];
-            }
-          }
-        }
-      } else {
-      // Items are strided by the block size, a multiple of the (power-of-two) pair count, so a
-      // thread always meets the same column pair l: it computes that one rotation per round and
-      // fetches the row pair's rotation from the lane that owns it (lane k of its own warp).
-      const int l = c.tid & mask;
-      int al = 0, bl = 0;
-      double cl = 1.0, sl = 0.0;
-      if (l < np) {
-        pair_of(rd, l, pp, al, bl);
-        const bool bigl = rotation(T, ld, al, bl, dim, cl, sl);
-        if (bigl && c.tid < np) *big = 1;
+      if (it.kind == 1) {
+        const double kaa = T[it.kaa], kbb = T[it.kbb], kab = T[it.kab];
+        const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+        const double xac = T[it.x0], xad = T[it.x1], xbc = T[it.x2], xbd = T[it.x3];
+        double ck, sk, cl, sl;
+        const bool bigk = rotation_of(kaa, kbb, kab, ck, sk);
+        (void)rotation_of(laa, lbb, lab, cl, sl);
+        if (it.diag && bigk) *big = 1;
+        const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+        const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+        Tn[it.z0] = cl * yac - sl * yad; Tn[it.z1] = sl * yac + cl * yad;
+        Tn[it.z2] = cl * ybc - sl * ybd; Tn[it.z3] = sl * ybc + cl * ybd;
+      } else if (it.kind == 2) {
+        const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+        const double va = J[it.x0], vb = J[it.x1];
+        double cl, sl;
+        (void)rotation_of(laa, lbb, lab, cl, sl);
+        Jn[it.z0] = cl * va - sl * vb;
+        Jn[it.z1] = sl * va + cl * vb;
       }
-      const int total = nblk + nrow;
-      for (int idx = c.tid; idx < ((total + 31) & ~31); idx += c.nt) {
-        const bool isblk = idx < nblk;
-        const int k = isblk ? (idx >> sh) : 0;
-        const double ck = __shfl_sync(0xffffffffu, cl, k);
-        const double sk = __shfl_sync(0xffffffffu, sl, k);
-        const int a = __shfl_sync(0xffffffffu, al, k);
-        const int b = __shfl_sync(0xffffffffu, bl, k);
-        if (idx >= total || l >= np) continue;
-        if (isblk) {
-          // 2x2 block (pair k rows, pair l columns) takes both rotations at once
-          const double xac = T[a * ld + al], xad = T[a * ld + bl], xbc = T[b * ld + al], xbd = T[b * ld + bl];
-          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
-          double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
-          double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
-          if (k == l && sk != 0.0) { zad = 0.0; zbc = 0.0; }
-          Tn[a * ld + al] = zac; Tn[a * ld + bl] = zad; Tn[b * ld + al] = zbc; Tn[b * ld + bl] = zbd;
-        } else if (sl != 0.0) {
-          const int x = (idx - nblk) >> sh;
-          const double va = J[x * ld + al], vb = J[x * ld + bl];
-          J[x * ld + al] = cl * va - sl * vb;
-          J[x * ld + bl] = sl * va + cl * vb;
-        }
-      }
-      }   // np <= 8
-#else
-      for (int idx = c.tid; idx < nblk + nrow; idx += c.nt) {
-        if (idx < nblk) {
-          // 2x2 block (pair k rows, pair l columns) takes both rotations at once
-          const int k = idx >> sh, l = idx & mask;
-          if (l >= np) continue;
-          int a, b, cc, d;
-          pair_of(rd, k, pp, a, b);
-          pair_of(rd, l, pp, cc, d);
-          double ck, sk, cl, sl;
-          const bool bigk = rotation(T, ld, a, b, dim, ck, sk);
-          if (k == l) { cl = ck; sl = sk; if (bigk) *big = 1; }
-          else (void)rotation(T, ld, cc, d, dim, cl, sl);
+      // further items (fewer threads than items): offsets on the fly
+      for (int idx = c.tid + c.nt; idx < total2; idx += c.nt) {
+        if (idx < nb2) {
+          const int k = idx / np, l = idx - k * np;
+          const int a = k, b = np + k, cc = l, d = np + l;
+          const double kaa = T[a * ld + a], kbb = T[b * ld + b], kab = T[a * ld + b];
+          const double laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
           const double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+          double ck, sk, cl, sl;
+          const bool bigk = rotation_of(kaa, kbb, kab, ck, sk);
+          (void)rotation_of(laa, lbb, lab, cl, sl);
+          if (k == l && bigk) *big = 1;
           const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
           const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
-          double zac = cl * yac - sl * yad, zad = sl * yac + cl * yad;
-          double zbc = cl * ybc - sl * ybd, zbd = sl * ybc + cl * ybd;
-          if (k == l && sk != 0.0) { zad = 0.0; zbc = 0.0; }
-          Tn[a * ld + cc] = zac; Tn[a * ld + d] = zad; Tn[b * ld + cc] = zbc; Tn[b * ld + d] = zbd;
+          const int pa = systolic_next(a, np), pb = systolic_next(b, np);
+          const int pc = systolic_next(cc, np), pd = systolic_next(d, np);
+          Tn[pa * ld + pc] = cl * yac - sl * yad; Tn[pa * ld + pd] = sl * yac + cl * yad;
+          Tn[pb * ld + pc] = cl * ybc - sl * ybd; Tn[pb * ld + pd] = sl * ybc + cl * ybd;
         } else {
-          const int q = idx - nblk;
-          const int x = q >> sh, k = q & mask;
-          if (k >= np) continue;
-          int a, b;
-          pair_of(rd, k, pp, a, b);
-          double ck, sk;
-          (void)rotation(T, ld, a, b, dim, ck, sk);
-          if (sk == 0.0) continue;
-          const double va = J[x * ld + a], vb = J[x * ld + b];
-          J[x * ld + a] = ck * va - sk * vb;
-          J[x * ld + b] = sk * va + ck * vb;
+          const int q = idx - nb2;
+          const int x = q / np, l = q - x * np;
+          const int cc = l, d = np + l;
+          const double laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
+          const double va = J[x * ld + cc], vb = J[x * ld + d];
+          double cl, sl;
+          (void)rotation_of(laa, lbb, lab, cl, sl);
+          Jn[x * ld + systolic_next(cc, np)] = cl * va - sl * vb;
+          Jn[x * ld + systolic_next(d, np)] = sl * va + cl * vb;
         }
       }
-#endif
       c.sync();
       { double* t = T; T = Tn; Tn = t; }
+      { double* t = J; J = Jn; Jn = t; }
     }
     const int again = *big;
     c.sync();
     if (!again) { ++sweep; break; }
   }
-  *Tio = T;
-  *Taltio = Tn;
+  *Tio = T; *Taltio = Tn; *Jio = J; *Jaltio = Jn;
   return sweep;
+}
+
+#ifndef FA_IRLS_HOST
+// More than 8 pairs, at most 32 (device only).  This thread's items are tid + u * nt: 2x2 blocks of T (kMT of
+// them) and (row, pair) items of J (kMJ).  Per item: the offset of its first element, the offsets
+// its results are stored at, and the pairs whose rotations it needs; offsets are below 2^16
+// (matrices of at most 64 x 65 doubles) and are kept two to a register.
+template <int kMT, int kMJ>
+FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
+                       int dim, int jrows) {
+  const int ld = s.ld;
+  const int pp = (dim + 1) & ~1;
+  const int np = pp >> 1;
+  double* T = *Tio;
+  double* Tn = *Taltio;
+  double* J = *Jio;
+  double* Jn = *Jaltio;
+  unsigned tdesc0[kMT], tdesc1[kMT], tdesc2[kMT], jdesc0[kMJ], jdesc1[kMJ];
+  bool tv[kMT], jv[kMJ];
+#pragma unroll
+  for (int u = 0; u < kMT; ++u) {
+    const int idx = c.tid + u * c.nt;
+    tv[u] = idx < np * np;
+    const int k = tv[u] ? idx / np : 0, l = tv[u] ? idx - k * np : 0;
+    const int pa = systolic_next(k, np) * ld, pb = systolic_next(np + k, np) * ld;
+    const int pc = systolic_next(l, np), pd = systolic_next(np + l, np);
+    tdesc0[u] = (unsigned)(k * ld + l) | ((unsigned)k << 16) | ((unsigned)l << 24);
+    tdesc1[u] = (unsigned)(pa + pc) | ((unsigned)(pa + pd) << 16);
+    tdesc2[u] = (unsigned)(pb + pc) | ((unsigned)(pb + pd) << 16);
+  }
+#pragma unroll
+  for (int u = 0; u < kMJ; ++u) {
+    const int idx = c.tid + u * c.nt;
+    jv[u] = idx < jrows * np;
+    const int x = jv[u] ? idx / np : 0, l = jv[u] ? idx - x * np : 0;
+    jdesc0[u] = (unsigned)(x * ld + l) | ((unsigned)l << 16);
+    jdesc1[u] = (unsigned)(x * ld + systolic_next(l, np)) | ((unsigned)(x * ld + systolic_next(np + l, np)) << 16);
+  }
+  int sweep = 0;
+  if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
+  c.sync();
+  for (; sweep < kMaxSweeps; ++sweep) {
+    int* big = &s.flags[(sweep & 1) ? 3 : 0];
+    if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
+    for (int rd = 0; rd < pp - 1; ++rd) {
+      // every warp works out all np <= 32 rotations itself, lane q the one of pair q; the items then
+      // fetch the two (one) they need with shuffles: no second barrier, no waiting for one warp
+      const int lane = c.tid & 31;
+      double x0[kMT], x1[kMT], x2[kMT], x3[kMT], v0[kMJ], v1[kMJ];
+#pragma unroll
+      for (int u = 0; u < kMT; ++u) {
+        if (tv[u]) {
+          const int tb = tdesc0[u] & 0xffffu;
+          x0[u] = T[tb]; x1[u] = T[tb + np]; x2[u] = T[tb + np * ld]; x3[u] = T[tb + np * ld + np];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kMJ; ++u) {
+        if (jv[u]) { const int jb = jdesc0[u] & 0xffffu; v0[u] = J[jb]; v1[u] = J[jb + np]; }
+      }
+      double cq = 1.0, sq = 0.0;
+      if (lane < np) {
+        const int o = lane * (ld + 1);
+        if (rotation_of(T[o], T[o + np * (ld + 1)], T[o + np], cq, sq) && c.tid < np) *big = 1;
+      }
+#pragma unroll
+      for (int u = 0; u < kMT; ++u) {
+        const int tk = (tdesc0[u] >> 16) & 0xffu, tl = tdesc0[u] >> 24;
+        const double ck = __shfl_sync(0xffffffffu, cq, tk), sk = __shfl_sync(0xffffffffu, sq, tk);
+        const double cl = __shfl_sync(0xffffffffu, cq, tl), sl = __shfl_sync(0xffffffffu, sq, tl);
+        if (tv[u]) {
+          const double yac = ck * x0[u] - sk * x2[u], yad = ck * x1[u] - sk * x3[u];
+          const double ybc = sk * x0[u] + ck * x2[u], ybd = sk * x1[u] + ck * x3[u];
+          Tn[tdesc1[u] & 0xffffu] = cl * yac - sl * yad; Tn[tdesc1[u] >> 16] = sl * yac + cl * yad;
+          Tn[tdesc2[u] & 0xffffu] = cl * ybc - sl * ybd; Tn[tdesc2[u] >> 16] = sl * ybc + cl * ybd;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kMJ; ++u) {
+        const int jl = jdesc0[u] >> 16;
+        const double cl = __shfl_sync(0xffffffffu, cq, jl), sl = __shfl_sync(0xffffffffu, sq, jl);
+        if (jv[u]) {
+          Jn[jdesc1[u] & 0xffffu] = cl * v0[u] - sl * v1[u];
+          Jn[jdesc1[u] >> 16] = sl * v0[u] + cl * v1[u];
+        }
+      }
+      if (lane < np) { s.rc[lane] = cq; s.rs[lane] = sq; }     // same values from every warp: for the loops below
+      // items beyond the per-thread lists (a smaller block than expected): offsets on the fly
+      if (kMT * c.nt < np * np || kMJ * c.nt < jrows * np) c.sync();
+      for (int idx = c.tid + kMT * c.nt; idx < np * np; idx += c.nt) {
+        const int k = idx / np, l = idx - k * np;
+        const int a = k, b = np + k, cc = l, d = np + l;
+        const double ck = s.rc[k], sk = s.rs[k], cl = s.rc[l], sl = s.rs[l];
+        const double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+        const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+        const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+        const int pa = systolic_next(a, np), pb = systolic_next(b, np);
+        const int pc = systolic_next(cc, np), pd = systolic_next(d, np);
+        Tn[pa * ld + pc] = cl * yac - sl * yad; Tn[pa * ld + pd] = sl * yac + cl * yad;
+        Tn[pb * ld + pc] = cl * ybc - sl * ybd; Tn[pb * ld + pd] = sl * ybc + cl * ybd;
+      }
+      for (int idx = c.tid + kMJ * c.nt; idx < jrows * np; idx += c.nt) {
+        const int x = idx / np, l = idx - x * np;
+        const int cc = l, d = np + l;
+        const double cl = s.rc[l], sl = s.rs[l];
+        const double va = J[x * ld + cc], vb = J[x * ld + d];
+        Jn[x * ld + systolic_next(cc, np)] = cl * va - sl * vb;
+        Jn[x * ld + systolic_next(d, np)] = sl * va + cl * vb;
+      }
+      c.sync();
+      { double* t = T; T = Tn; Tn = t; }
+      { double* t = J; J = Jn; Jn = t; }
+    }
+    const int again = *big;
+    c.sync();
+    if (!again) { ++sweep; break; }
+  }
+  *Tio = T; *Taltio = Tn; *Jio = J; *Jaltio = Jn;
+  return sweep;
+}
+#endif
+
+template <bool LARGE>
+FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio, int dim,
+                 int jrows) {
+  if (dim < 2) return 0;
+#ifndef FA_IRLS_HOST
+  // item slots per thread are compile-time (slots without an item still cost their instructions):
+  // one of each up to 16 pairs with 512 threads, two blocks and four J items up to 32 pairs
+  const int np = (dim + 1) >> 1;
+  if (LARGE && np > 8) {
+    if (np * np <= c.nt && jrows * np <= c.nt) return jacobi_large<1, 1>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
+    return jacobi_large<2, 4>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
+  }
+#endif
+  return jacobi_small(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
 }
 
 // ev[k] = T[k][k]; ord[q] = index of the q-th largest (ties by index).  All threads return
@@ -802,7 +915,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       if (a >= r || b >= r) s.T[a * ld + b] = 0.0;
     }
     c.sync();
-    sw = jacobi<LARGE>(c, s, &s.T, &s.tmp, s.J, r, r);
+    sw = jacobi<LARGE>(c, s, &s.T, &s.tmp, &s.J, &s.M, r, r);   // M is free until the next weights
     if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
     m_eff = sort_eigs(c, s, s.T, r, m);
 
