@@ -219,8 +219,8 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
   double* Jn = *Jaltio;
   const int nb2 = np * np, total2 = nb2 + jrows * np;
   // the item this thread owns for the whole solve (element offsets into T / J)
-  struct Item { int kind, diag, kaa, kbb, kab, laa, lbb, lab, x0, x1, x2, x3, z0, z1, z2, z3; } it;
-  it.kind = 0;
+  struct Item { int kind, diag, ksrc, kaa, kbb, kab, laa, lbb, lab, x0, x1, x2, x3, z0, z1, z2, z3; } it;
+  it.kind = 0; it.ksrc = -1; it.laa = it.lbb = it.lab = 0;
   {
     const int idx = c.tid;
     if (idx < nb2) {
@@ -232,6 +232,14 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       it.laa = cc * ld + cc; it.lbb = d * ld + d; it.lab = cc * ld + d;
       it.x0 = a * ld + cc; it.x1 = a * ld + d; it.x2 = b * ld + cc; it.x3 = b * ld + d;
       it.z0 = pa * ld + pc; it.z1 = pa * ld + pd; it.z2 = pb * ld + pc; it.z3 = pb * ld + pd;
+#ifndef FA_IRLS_HOST
+      // a lane of this warp whose own (column) pair is k hands over the row rotation
+      const int w0 = idx & ~31;
+      for (int j = 0; j < 32; ++j) {
+        const int o = w0 + j;
+        if (o < total2 && (o < nb2 ? o % np : (o - nb2) % np) == k) { it.ksrc = j; break; }
+      }
+#endif
     } else if (idx < total2) {
       const int q = idx - nb2;
       const int x = q / np, l = q - x * np;
@@ -251,6 +259,34 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
     int* big = &s.flags[(sweep & 1) ? 3 : 0];
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
+#ifndef FA_IRLS_HOST
+      {
+        // every lane with an item works out the rotation of its column pair l; a block of T gets
+        // its row rotation from the lane `ksrc` of its warp (worked out here only if there is none)
+        double cl = 1.0, sl = 0.0;
+        bool bigl = false;
+        double xac = 0.0, xad = 0.0, xbc = 0.0, xbd = 0.0;
+        if (it.kind != 0) {
+          const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+          if (it.kind == 1) { xac = T[it.x0]; xad = T[it.x1]; xbc = T[it.x2]; xbd = T[it.x3]; }
+          else { xac = J[it.x0]; xad = J[it.x1]; }
+          bigl = rotation_of(laa, lbb, lab, cl, sl);
+        }
+        const int src = it.ksrc < 0 ? 0 : it.ksrc;
+        double ck = __shfl_sync(0xffffffffu, cl, src), sk = __shfl_sync(0xffffffffu, sl, src);
+        if (it.kind == 1) {
+          if (it.ksrc < 0) (void)rotation_of(T[it.kaa], T[it.kbb], T[it.kab], ck, sk);
+          if (it.diag && bigl) *big = 1;
+          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+          Tn[it.z0] = cl * yac - sl * yad; Tn[it.z1] = sl * yac + cl * yad;
+          Tn[it.z2] = cl * ybc - sl * ybd; Tn[it.z3] = sl * ybc + cl * ybd;
+        } else if (it.kind == 2) {
+          Jn[it.z0] = cl * xac - sl * xad;
+          Jn[it.z1] = sl * xac + cl * xad;
+        }
+      }
+#else
       if (it.kind == 1) {
         const double kaa = T[it.kaa], kbb = T[it.kbb], kab = T[it.kab];
         const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
@@ -271,6 +307,7 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
         Jn[it.z0] = cl * va - sl * vb;
         Jn[it.z1] = sl * va + cl * vb;
       }
+#endif
       // further items (fewer threads than items): offsets on the fly
       for (int idx = c.tid + c.nt; idx < total2; idx += c.nt) {
         if (idx < nb2) {
@@ -722,10 +759,24 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   for (int k = 0; k < p; ++k) {
     int piv = -1;
     double dmax = kRankRel;
-    for (int j = 0; j < p; ++j) {                 // every thread scans; ties go to the lowest index
+#ifndef FA_IRLS_HOST
+    // every warp finds the pivot itself (two candidates per lane, butterfly); ties go to the lowest index
+    for (int j = (c.tid & 31); j < p; j += 32) {
       const double dj = s.u[j];
       if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
     }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const double od = __shfl_xor_sync(0xffffffffu, dmax, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, piv, off);
+      if (od > dmax || (od == dmax && oi >= 0 && (piv < 0 || oi < piv))) { dmax = od; piv = oi; }
+    }
+#else
+    for (int j = 0; j < p; ++j) {                 // ties go to the lowest index
+      const double dj = s.u[j];
+      if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
+    }
+#endif
     if (piv < 0) break;
     const double rkk = sqrt(dmax), rinv = 1.0 / rkk;
     for (int j = c.tid; j < p; j += c.nt) {
