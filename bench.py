@@ -143,7 +143,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     from oracle import fa_oracle as fo
-    n_sample = max(4096, w.n // 64)
+    n_sample = max(4096, min(w.n // 64, int(10.0 / (2.7e-9 * w.p * w.p * w.iters))))   # about 10 s of oracle time per step
     ws = w.scaled(n_sample)
     G = si.to_float64(si.generate(ws))
     for _ in range(args.warmup):
@@ -323,7 +323,8 @@ def main():
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        n_sample = max(4096, w.n // 8)
+        # about 20 s of oracle time: its cost grows like n * p^2 * rounds (2.7e-9 s per unit on this class of host)
+        n_sample = max(4096, min(w.n // 8, int(20.0 / (2.7e-9 * w.p * w.p * w.iters))))
         t_s = time_oracle(w, n_sample)
         scale = w.n / n_sample
         cpu = {"value": 1.0 / (t_s * scale), "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libfa_b200.so")
-SOURCES = ["fa_api.cu", "fa_gram.cu", "fa_irls.cu", "fa_combine.cu", "fa_static.cu", "fa_gram_tc.cu"]
+SOURCES = ["fa_api.cu", "fa_gram.cu", "fa_irls.cu", "fa_combine.cu", "fa_static.cu", "fa_gram_tc.cu", "fa_gram_tm.cu"]
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
     "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr",

@@ -469,6 +469,7 @@ size_t gram_partials_bytes(int p, long long n, int dtype) {
 cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
                         double* K, int* status, cudaStream_t st) {
   if (gram_tc_eligible(G, dtype, p, n)) return launch_gram_tc(G, p, n, partials, counter, K, status, st);
+  if (gram_tm_eligible(G, dtype, p, n)) return launch_gram_tm(G, dtype, p, n, partials, counter, K, status, st);
   const gram::Shape sh = gram::pick_shape(p);
   const int S = dtype == 0 ? 4 : 2;
   gram::Params prm{};

@@ -1,0 +1,349 @@
+// Gram pass fed by TMA TENSOR loads (K_ij = <g_i, g_j>, Section 2.1) -- the fast path of fa_gram
+// whenever the matrix starts on a 16-byte boundary.
+//
+// One tensor-map load brings a 256-column tile of ALL rows of a row class into shared memory
+// (15-64 KB per instruction).  Measured on B200 this feed sustains about 24.7 bytes per clock and SM
+// (7.2 TB/s), against 19.5 for one 1-D bulk copy of 4 KB per row (fa_gram.cu) -- the tensor unit
+// pays its fixed cost per ROW of a box, and 1 KB rows are long enough.
+//
+// Row classes.  A tensor map wants every row to start on a 16-byte boundary (base and strides are
+// multiples of 16 bytes), and n * sizeof(T) need not be one.  So the rows are split into q classes
+// i mod q (q = 1, 2 or 4: the smallest with q * n * sizeof(T) a multiple of 16); class c gets its own
+// map over the rows c, c + q, ... with stride q * n, based at the 16-byte boundary at or before the
+// start of row c.  Row c therefore begins `shift_c` elements into its map's rows, the tile of a
+// class is read back with that shift, and consecutive tiles advance by 256 - 16/sizeof(T) columns
+// instead of 256 so that every class holds all the columns of a tile (1.6 % re-read; none when
+// q = 1).  Columns past the end of a row are outside the map's extent and arrive as zeros, so
+// there is no ragged tile; the few elements before row c that the shift drags in belong to row
+// c - 1 and are never read back.
+//
+// p <= 16: every warp takes whole tiles (tile u of a block goes to warp u mod 12) and loads them
+// itself; every thread keeps the upper triangle for its columns, as in fa_gram.cu; products in
+// fp32, runs of at most 64 columns, warp butterfly into fp64.  Block totals and the last-block reduction are
+// the ones of fa_gram.cu (bit-reproducible, single launch).
+#include <cuda.h>
+
+#include "fa_common.cuh"
+#include "fa_gram_finish.cuh"
+#include "fa_kernels.h"
+
+namespace fa {
+namespace gramtm {
+
+constexpr int kTileCols = 256;               // box width in elements
+constexpr int kMaxClasses = 4;
+constexpr int kFlushCols = 64;               // fp32 running sums cover at most this many columns
+constexpr int kTriWarps = 12;                // p <= 16: 12 warps, 168 registers each
+constexpr int kMaxDepth = 4;                 // stages per warp
+constexpr size_t kStageBudget = 184 * 1024;  // bytes of shared memory for all stages
+
+struct Maps { CUtensorMap map[kMaxClasses]; };
+
+struct Layout {
+  int depth;                   // stages per warp
+  int q;                       // row classes
+  int step;                    // columns a tile advances by
+  int rows[kMaxClasses];       // rows in class c
+  int rowbase[kMaxClasses];    // staged row index of the first row of class c
+  int shift[kMaxClasses];      // elements between the map's row start and the row's own start
+};
+
+struct Params {
+  int p;
+  long long num_tiles;
+  double* partials;            // [p(p+1)/2][gridDim.x]
+  unsigned int* counter;
+  double* K;
+  int* status;
+};
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+template <int NACCP, int L, int MASK>
+__device__ __forceinline__ void butterfly_step(float (&x)[NACCP], int lane) {
+  if constexpr (MASK >= 1) {
+    constexpr int H = L / 2;
+    const bool up = (lane & MASK) != 0;
+#pragma unroll
+    for (int k = 0; k < H; ++k) {
+      float lo = x[k], hi = x[H + k];
+      float send = up ? lo : hi;
+      float keep = up ? hi : lo;
+      x[k] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
+    }
+    butterfly_step<NACCP, H, MASK / 2>(x, lane);
+  }
+}
+
+// Reduce-scatter of NACCP values per lane over the warp, then into the lane's fp64 sums.
+template <int NACCP>
+__device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP / 32], int lane) {
+  butterfly_step<NACCP, NACCP, 16>(acc, lane);
+#pragma unroll
+  for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
+#pragma unroll
+  for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
+}
+
+// p <= 16.  No producer: every warp owns `depth` stages and keeps them loaded itself -- lane 0 issues
+// the tensor loads of the warp's next tile into the stage the warp has just finished with.  (One
+// issuing thread for the whole block could not keep up: a tile costs it about 500 cycles, and a
+// stage must in any case be consumed by the warp that waited for its previous phases -- a parity
+// wait cannot tell "two phases behind" from "done".)  Tile u of a block (global tile
+// blockIdx.x + u * gridDim.x) goes to warp u mod 12.
+template <typename T, int V, int PB>
+__global__ void __launch_bounds__(kTriWarps * 32, 1)
+gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const Layout lay) {
+  constexpr int S = sizeof(T);
+  constexpr int kThreads = kTriWarps * 32;
+  constexpr int NACC = PB * (PB + 1) / 2;
+  constexpr int NACCP = (NACC + 31) / 32 * 32;
+  extern __shared__ __align__(1024) char smem[];
+  const int stage_bytes = prm.p * kTileCols * S;
+  const int depth = lay.depth;
+  char* stages = smem;
+  double* totals = reinterpret_cast<double*>(smem + (size_t)kTriWarps * depth * stage_bytes);
+  uint64_t* full = reinterpret_cast<uint64_t*>(totals + kTriWarps * NACCP);
+  int* flag = reinterpret_cast<int*>(full + kTriWarps * kMaxDepth);      // last-block flag
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    for (int s = 0; s < kTriWarps * kMaxDepth; ++s) mbar_init(&full[s], 1);
+  }
+  fence_proxy_async();
+  __syncthreads();
+
+  float acc[NACCP];
+  double dacc[NACCP / 32];
+#pragma unroll
+  for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
+#pragma unroll
+  for (int k = 0; k < NACCP / 32; ++k) dacc[k] = 0.0;
+  int rowoff[PB];
+#pragma unroll
+  for (int i = 0; i < PB; ++i) {
+    const int ii = i < prm.p ? i : 0;
+    const int cidx = ii % lay.q;
+    rowoff[i] = (lay.rowbase[cidx] + ii / lay.q) * (kTileCols * S) + lay.shift[cidx] * S;
+  }
+  char* mystages = stages + (size_t)warp * depth * stage_bytes;
+  uint64_t* mybars = full + warp * kMaxDepth;
+
+  // v-th tile of this warp: global tile blockIdx.x + (warp + v * 12) * gridDim.x, stage v mod depth
+  auto tile_of = [&](long long v) { return (long long)blockIdx.x + ((long long)warp + v * kTriWarps) * gridDim.x; };
+  auto issue = [&](long long v) {       // lane 0 only
+    const long long t = tile_of(v);
+    if (t >= prm.num_tiles) return;
+    const int s = static_cast<int>(v % depth);
+    mbar_arrive_expect_tx(&mybars[s], static_cast<uint32_t>(stage_bytes));
+    char* sbase = mystages + (size_t)s * stage_bytes;
+    const int x0 = static_cast<int>(t * lay.step);
+    for (int cidx = 0; cidx < lay.q; ++cidx)
+      if (lay.rows[cidx] > 0)
+        tma_load_2d(sbase + (size_t)lay.rowbase[cidx] * kTileCols * S, &maps.map[cidx], x0, 0, &mybars[s]);
+  };
+  if (lane == 0)
+    for (int v = 0; v < depth; ++v) issue(v);
+
+  const int groups = lay.step / V;
+  const int per_tile = (groups + 31) / 32 * V;      // columns a thread takes from one tile
+  int since = 0;
+  for (long long v = 0;; ++v) {
+    if (tile_of(v) >= prm.num_tiles) break;
+    const int s = static_cast<int>(v % depth);
+    if (!mbar_wait(&mybars[s], static_cast<uint32_t>((v / depth) & 1))) {
+      if (lane == 0) {
+        if (prm.status) atomicOr(prm.status, kStTimeout);
+        // let this warp's other loads land before the block can exit
+        for (long long w = v + 1; w < v + depth; ++w)
+          if (tile_of(w) < prm.num_tiles) (void)mbar_wait(&mybars[w % depth], static_cast<uint32_t>((w / depth) & 1));
+      }
+      break;
+    }
+    const char* sbase = mystages + (size_t)s * stage_bytes;
+    for (int cg = lane; cg < groups; cg += 32) {
+      float x[PB][V];
+#pragma unroll
+      for (int i = 0; i < PB; ++i) {
+        SmemVec<T, V>::load(sbase + rowoff[i] + cg * (V * S), x[i]);
+        if (i >= prm.p) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) x[i][e] = 0.f;
+        }
+      }
+      int idx = 0;
+#pragma unroll
+      for (int i = 0; i < PB; ++i)
+#pragma unroll
+        for (int j = i; j < PB; ++j) {
+#pragma unroll
+          for (int e = 0; e < V; ++e) acc[idx] = fmaf(x[i][e], x[j][e], acc[idx]);
+          ++idx;
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+      fence_proxy_async();          // the warp's reads of this stage come before the next load's writes
+      issue(v + depth);
+    }
+    since += per_tile;
+    if (since + per_tile > kFlushCols) { flush<NACCP>(acc, dacc, lane); since = 0; }
+  }
+  flush<NACCP>(acc, dacc, lane);
+#pragma unroll
+  for (int k = 0; k < NACCP / 32; ++k) totals[warp * NACCP + lane * (NACCP / 32) + k] = dacc[k];
+  __syncthreads();
+
+  // block total (fixed warp order) -> this block's entries, then the last block forms K
+  for (int e = tid; e < NACC; e += kThreads) {
+    int i = 0, r = e;
+    while (r >= PB - i) { r -= PB - i; ++i; }
+    const int j = i + r;
+    if (j < prm.p) {
+      double sum = 0.0;
+      for (int w = 0; w < kTriWarps; ++w) sum += totals[w * NACCP + e];
+      prm.partials[(size_t)gram::canon_index(i, j, prm.p) * gridDim.x + blockIdx.x] = sum;
+    }
+  }
+  gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
+}
+
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Row classes of a p x n matrix of S-byte elements: 0 when more than kMaxClasses would be needed.
+int class_count(long long n, int S) {
+  for (int q = 1; q <= kMaxClasses; q *= 2)
+    if ((static_cast<unsigned long long>(q) * static_cast<unsigned long long>(n) * S) % 16 == 0) return q;
+  return 0;
+}
+
+bool build(const void* G, int dtype, int p, long long n, Maps& maps, Layout& lay) {
+  EncodeTiledFn enc = encode_tiled();
+  const int S = dtype == 0 ? 4 : 2;
+  const int q = class_count(n, S);
+  if (!enc || q == 0) return false;
+  lay.q = q;
+  lay.step = q == 1 ? kTileCols : kTileCols - 16 / S;
+  int base = 0;
+  for (int c = 0; c < kMaxClasses; ++c) { lay.rows[c] = 0; lay.rowbase[c] = 0; lay.shift[c] = 0; }
+  for (int c = 0; c < q; ++c) {
+    const int rows = c < p ? (p - c + q - 1) / q : 0;
+    lay.rows[c] = rows;
+    lay.rowbase[c] = base;
+    base += rows;
+    if (rows == 0) continue;
+    const unsigned long long off = static_cast<unsigned long long>(c) * static_cast<unsigned long long>(n) * S;   // bytes
+    const int skew = static_cast<int>(off % 16);
+    lay.shift[c] = skew / S;
+    const char* start = static_cast<const char*>(G) + off - skew;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(n) + static_cast<cuuint64_t>(lay.shift[c]),
+                                static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(q) * static_cast<cuuint64_t>(n) * S};
+    const cuuint32_t box[2] = {kTileCols, static_cast<cuuint32_t>(rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&maps.map[c], dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+            const_cast<char*>(start), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return false;
+  }
+  return true;
+}
+
+template <typename K>
+cudaError_t launch(K kernel, const Maps& maps, const Params& prm, const Layout& lay, int grid, int threads,
+                   size_t smem, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kernel<<<grid, threads, smem, st>>>(maps, prm, lay);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t dispatch_tri(int pb, int vec, const Maps& maps, const Params& prm, const Layout& lay, int grid, size_t smem,
+                         cudaStream_t st) {
+#define FA_TM_CASE(PB)                                                                                       \
+  case PB:                                                                                                   \
+    return vec == 2 ? launch(gram_tri_tm_kernel<T, 2, PB>, maps, prm, lay, grid, kTriWarps * 32, smem, st) \
+                    : launch(gram_tri_tm_kernel<T, 1, PB>, maps, prm, lay, grid, kTriWarps * 32, smem, st);
+  switch (pb) {
+    FA_TM_CASE(4)
+    FA_TM_CASE(8)
+    FA_TM_CASE(12)
+    FA_TM_CASE(15)
+    FA_TM_CASE(16)
+  }
+#undef FA_TM_CASE
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace
+}  // namespace gramtm
+
+// Tensor-load feed: matrix on a 16-byte boundary, at most four row classes, enough columns for a
+// few tiles per block, column coordinates within the 32-bit range of the copy instruction.
+bool gram_tm_eligible(const void* G, int dtype, int p, long long n) {
+  const int S = dtype == 0 ? 4 : 2;
+  return p >= 1 && p <= 16 && (reinterpret_cast<uintptr_t>(G) % 16) == 0 && n >= 4096 && n < (1LL << 31) - 4096 &&
+         gramtm::class_count(n, S) != 0 && gramtm::encode_tiled() != nullptr;
+}
+
+cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
+                           double* K, int* status, cudaStream_t st) {
+  gramtm::Maps maps;
+  gramtm::Layout lay;
+  if (!gramtm::build(G, dtype, p, n, maps, lay)) return cudaErrorInvalidValue;
+  const int S = dtype == 0 ? 4 : 2;
+  gramtm::Params prm{};
+  prm.p = p;
+  prm.num_tiles = (n + lay.step - 1) / lay.step;
+  prm.partials = partials;
+  prm.counter = counter;
+  prm.K = K;
+  prm.status = status;
+  const int sms = sm_count();
+  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
+  cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
+  if (e != cudaSuccess) return e;
+  const int pb = p <= 4 ? 4 : p <= 8 ? 8 : p <= 12 ? 12 : p <= 15 ? 15 : 16;
+  const int naccp = (pb * (pb + 1) / 2 + 31) / 32 * 32;
+  // two elements per shared load when every class's shift is even
+  bool even = true;
+  for (int c = 0; c < lay.q; ++c) even = even && (lay.shift[c] % 2 == 0);
+  const int vec = even ? 2 : 1;
+  const size_t stage_bytes = (size_t)p * gramtm::kTileCols * S;
+  int depth = (int)(gramtm::kStageBudget / (gramtm::kTriWarps * stage_bytes));
+  depth = depth < 1 ? 1 : depth > gramtm::kMaxDepth ? gramtm::kMaxDepth : depth;
+  lay.depth = depth;
+  const size_t smem = (size_t)gramtm::kTriWarps * depth * stage_bytes + (size_t)gramtm::kTriWarps * naccp * sizeof(double) +
+                      (size_t)gramtm::kTriWarps * gramtm::kMaxDepth * sizeof(uint64_t) + 64;
+  if (dtype == 0) return gramtm::dispatch_tri<float>(pb, vec, maps, prm, lay, grid, smem, st);
+  return gramtm::dispatch_tri<__nv_bfloat16>(pb, vec, maps, prm, lay, grid, smem, st);
+}
+
+}  // namespace fa

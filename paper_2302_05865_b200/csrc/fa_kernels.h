@@ -19,6 +19,11 @@ bool gram_tc_eligible(const void* G, int dtype, int p, long long n);
 cudaError_t launch_gram_tc(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
                            int* status, cudaStream_t st);
 
+// Gram pass fed by tensor loads (matrix on a 16-byte boundary, p <= 16); same scratch and output.
+bool gram_tm_eligible(const void* G, int dtype, int p, long long n);
+cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
+                           double* K, int* status, cudaStream_t st);
+
 // Persistent single-block IRLS on K (p x p).
 struct IrlsArgs {
   const double* K;
