@@ -21,32 +21,12 @@
 // itself; every thread keeps the upper triangle for its columns, as in fa_gram.cu; products in
 // fp32, runs of at most 64 columns, warp butterfly into fp64.  Block totals and the last-block reduction are
 // the ones of fa_gram.cu (bit-reproducible, single launch).
-#include <cuda.h>
-
-#include "fa_common.cuh"
+#include "fa_gram_tm.cuh"
 #include "fa_gram_finish.cuh"
 #include "fa_kernels.h"
 
 namespace fa {
 namespace gramtm {
-
-constexpr int kTileCols = 256;               // box width in elements
-constexpr int kMaxClasses = 4;
-constexpr int kFlushCols = 64;               // fp32 running sums cover at most this many columns
-constexpr int kTriWarps = 12;                // p <= 16: 12 warps, 168 registers each
-constexpr int kMaxDepth = 4;                 // stages per warp
-constexpr size_t kStageBudget = 184 * 1024;  // bytes of shared memory for all stages
-
-struct Maps { CUtensorMap map[kMaxClasses]; };
-
-struct Layout {
-  int depth;                   // stages per warp
-  int q;                       // row classes
-  int step;                    // columns a tile advances by
-  int rows[kMaxClasses];       // rows in class c
-  int rowbase[kMaxClasses];    // staged row index of the first row of class c
-  int shift[kMaxClasses];      // elements between the map's row start and the row's own start
-};
 
 struct Params {
   int p;
@@ -56,14 +36,6 @@ struct Params {
   double* K;
   int* status;
 };
-
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          smem_u32(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
-}
 
 template <int NACCP, int L, int MASK>
 __device__ __forceinline__ void butterfly_step(float (&x)[NACCP], int lane) {
@@ -242,6 +214,8 @@ int class_count(long long n, int S) {
   return 0;
 }
 
+}  // namespace
+
 bool build(const void* G, int dtype, int p, long long n, Maps& maps, Layout& lay) {
   EncodeTiledFn enc = encode_tiled();
   const int S = dtype == 0 ? 4 : 2;
@@ -274,6 +248,13 @@ bool build(const void* G, int dtype, int p, long long n, Maps& maps, Layout& lay
   }
   return true;
 }
+
+bool available(const void* G, int dtype, long long n) {
+  return (reinterpret_cast<uintptr_t>(G) % 16) == 0 && n >= 4096 && n < (1LL << 31) - 4096 &&
+         class_count(n, dtype == 0 ? 4 : 2) != 0 && encode_tiled() != nullptr;
+}
+
+namespace {
 
 template <typename K>
 cudaError_t launch(K kernel, const Maps& maps, const Params& prm, const Layout& lay, int grid, int threads,
@@ -308,9 +289,7 @@ cudaError_t dispatch_tri(int pb, int vec, const Maps& maps, const Params& prm, c
 // Tensor-load feed: matrix on a 16-byte boundary, at most four row classes, enough columns for a
 // few tiles per block, column coordinates within the 32-bit range of the copy instruction.
 bool gram_tm_eligible(const void* G, int dtype, int p, long long n) {
-  const int S = dtype == 0 ? 4 : 2;
-  return p >= 1 && p <= 16 && (reinterpret_cast<uintptr_t>(G) % 16) == 0 && n >= 4096 && n < (1LL << 31) - 4096 &&
-         gramtm::class_count(n, S) != 0 && gramtm::encode_tiled() != nullptr;
+  return p >= 1 && p <= 16 && gramtm::available(G, dtype, n);
 }
 
 cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
