@@ -32,7 +32,24 @@ __device__ __forceinline__ void finish_gram(double* partials, unsigned int* coun
     double sum[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) sum[e] = 0.0;
-    for (int b = lane; b < nb; b += 32) {
+    // the first 160 blocks: all loads of a lane go out before the first add (same order of adds)
+    constexpr int kUnrolled = 5;
+    double v[kUnrolled][E];
+#pragma unroll
+    for (int k = 0; k < kUnrolled; ++k) {
+      const int b = lane + 32 * k;
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+        v[k][e] = (b < nb && c0 + e < ntri) ? __ldcg(partials + (size_t)(c0 + e) * nb + b) : 0.0;
+    }
+#pragma unroll
+    for (int k = 0; k < kUnrolled; ++k) {
+      const int b = lane + 32 * k;
+#pragma unroll
+      for (int e = 0; e < E; ++e)
+        if (b < nb && c0 + e < ntri) sum[e] += v[k][e];
+    }
+    for (int b = lane + 32 * kUnrolled; b < nb; b += 32) {
 #pragma unroll
       for (int e = 0; e < E; ++e)
         if (c0 + e < ntri) sum[e] += __ldcg(partials + (size_t)(c0 + e) * nb + b);
