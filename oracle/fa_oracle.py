@@ -21,7 +21,7 @@ What it computes (Flag Aggregator paper, arXiv 2302.05865):
 How each round is taken (the paper names the procedure but prints no update
 formula; this is the reading used, each item listed in the design notes):
 
-  * round 1 uses uniform weights, so it is PCA of the gradient matrix
+  * the first round uses uniform weights, so it is PCA of the gradient matrix
     (appendix "Experiments with other Byzantine attacks or baselines");
   * later rounds reweight every square-root term of the objective by
     1 / (normaliser * sqrt(term's current value)) -- for the data terms this
