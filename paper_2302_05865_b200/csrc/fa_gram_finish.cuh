@@ -27,27 +27,28 @@ __device__ __forceinline__ void finish_gram(double* partials, unsigned int* coun
   const int ntri = p * (p + 1) / 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   const int nb = gridDim.x;
-  constexpr int E = 8;                           // entries a warp sums at once (independent loads in flight)
+  constexpr int E = 10;                          // entries a warp sums at once
   for (int c0 = warp * E; c0 < ntri; c0 += nwarps * E) {
     double sum[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) sum[e] = 0.0;
-    // the first 160 blocks: all loads of a lane go out before the first add (same order of adds)
+    // The first 160 blocks: every load of the lane goes out before the first add -- the loads are
+    // unconditional (clamped indices, masked afterwards) so that nothing keeps them from being issued
+    // back to back; a round then costs one trip to L2 (about 0.7 us here) instead of five.  The adds
+    // keep their order (blocks lane, lane + 32, ...), so the sums are the same bits as before.
     constexpr int kUnrolled = 5;
     double v[kUnrolled][E];
 #pragma unroll
     for (int k = 0; k < kUnrolled; ++k) {
-      const int b = lane + 32 * k;
+      const int b = min(lane + 32 * k, nb - 1);
 #pragma unroll
-      for (int e = 0; e < E; ++e)
-        v[k][e] = (b < nb && c0 + e < ntri) ? __ldcg(partials + (size_t)(c0 + e) * nb + b) : 0.0;
+      for (int e = 0; e < E; ++e) v[k][e] = __ldcg(partials + (size_t)min(c0 + e, ntri - 1) * nb + b);
     }
 #pragma unroll
     for (int k = 0; k < kUnrolled; ++k) {
-      const int b = lane + 32 * k;
+      const bool ok = lane + 32 * k < nb;
 #pragma unroll
-      for (int e = 0; e < E; ++e)
-        if (b < nb && c0 + e < ntri) sum[e] += v[k][e];
+      for (int e = 0; e < E; ++e) sum[e] += ok ? v[k][e] : 0.0;
     }
     for (int b = lane + 32 * kUnrolled; b < nb; b += 32) {
 #pragma unroll
