@@ -186,6 +186,144 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
   gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
 }
 
+// ---- 16 < p <= 32, one row class (rows on 16-byte boundaries), fp32.
+// The 32 x 32 triangle is cut into four parts of at most 136 sums -- the triangles of rows 0-15 and
+// 16-31 and the two 8 x 16 halves of the rectangle between them -- and a TEAM of four warps, one per
+// part, works through a tile together; the block's two teams take alternate tiles, each with its
+// own stages, and the first lane of a team re-issues the team's next load once the four warps have
+// met at the team's barrier.  Eight warps (two per scheduler) leave 255 registers per thread: the
+// sums, two columns of operands and nothing spilled.  Staged rows are exactly 1 KB apart, so every
+// shared load is one base register plus an immediate; rows p..31 of a stage are zeroed once and
+// never written.
+constexpr int kQuadWarps = 8;
+constexpr int kQuadDepth = 3;                // stages per team: 2 x 3 x 32 KB
+constexpr int kQuadAcc = 160;                // 136 rounded up to a multiple of 32
+
+__device__ __forceinline__ void team_barrier(int team) {
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(128) : "memory");
+}
+
+__global__ void __launch_bounds__(kQuadWarps * 32, 1)
+gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
+  constexpr int kThreads = kQuadWarps * 32;
+  constexpr int kRowBytes = kTileCols * 4;
+  constexpr int kStageBytes = 32 * kRowBytes;
+  extern __shared__ __align__(1024) char smem[];
+  char* stages = smem;
+  double* totals = reinterpret_cast<double*>(smem + (size_t)2 * kQuadDepth * kStageBytes);
+  uint64_t* full = reinterpret_cast<uint64_t*>(totals + kQuadWarps * kQuadAcc);
+  int* flag = reinterpret_cast<int*>(full + 2 * kQuadDepth);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int team = warp >> 2, role = warp & 3;
+
+  for (int i = tid * 16; i < 2 * kQuadDepth * kStageBytes; i += kThreads * 16)
+    *reinterpret_cast<uint4*>(stages + i) = make_uint4(0, 0, 0, 0);
+  if (tid == 0)
+    for (int s = 0; s < 2 * kQuadDepth; ++s) mbar_init(&full[s], 1);
+  fence_proxy_async();
+  __syncthreads();
+
+  char* mystages = stages + (size_t)team * kQuadDepth * kStageBytes;
+  uint64_t* mybars = full + team * kQuadDepth;
+  const uint32_t tile_bytes = static_cast<uint32_t>(prm.p * kRowBytes);
+  // v-th tile of this team: the block's tile 2 v + team, i.e. global tile blockIdx.x + (2 v + team) * gridDim.x
+  auto tile_of = [&](long long v) { return (long long)blockIdx.x + (2 * v + team) * (long long)gridDim.x; };
+  auto issue = [&](long long v) {       // first lane of the team only
+    const long long t = tile_of(v);
+    if (t >= prm.num_tiles) return;
+    const int s = static_cast<int>(v % kQuadDepth);
+    mbar_arrive_expect_tx(&mybars[s], tile_bytes);
+    tma_load_2d(mystages + (size_t)s * kStageBytes, &maps.map[0], static_cast<int>(t * kTileCols), 0, &mybars[s]);
+  };
+  const bool issuer = role == 0 && lane == 0;
+  if (issuer)
+    for (int v = 0; v < kQuadDepth; ++v) issue(v);
+
+  float acc[kQuadAcc];
+  double dacc[kQuadAcc / 32];
+#pragma unroll
+  for (int k = 0; k < kQuadAcc; ++k) acc[k] = 0.f;
+#pragma unroll
+  for (int k = 0; k < kQuadAcc / 32; ++k) dacc[k] = 0.0;
+  const int rowbase = (role < 2 ? 16 * role : 8 * (role - 2)) * kRowBytes;   // first row of the part (rectangle: its a-rows)
+  int since = 0;
+  for (long long v = 0;; ++v) {
+    if (tile_of(v) >= prm.num_tiles) break;
+    const int s = static_cast<int>(v % kQuadDepth);
+    if (!mbar_wait(&mybars[s], static_cast<uint32_t>((v / kQuadDepth) & 1))) {
+      if (lane == 0 && prm.status) atomicOr(prm.status, kStTimeout);
+      break;
+    }
+    const char* sbase = mystages + (size_t)s * kStageBytes;
+    if (role < 2) {
+#pragma unroll 1
+      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+        const char* ptr = sbase + rowbase + cg * 8;
+        float x[16][2];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) SmemVec<float, 2>::load(ptr + i * kRowBytes, x[i]);
+        int idx = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+#pragma unroll
+          for (int j = i; j < 16; ++j) {
+            acc[idx] = fmaf(x[i][0], x[j][0], acc[idx]);
+            acc[idx] = fmaf(x[i][1], x[j][1], acc[idx]);
+            ++idx;
+          }
+      }
+    } else {
+#pragma unroll 1
+      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+        const char* pa = sbase + rowbase + cg * 8;
+        const char* pb = sbase + 16 * kRowBytes + cg * 8;
+        float a[8][2], b[16][2];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) SmemVec<float, 2>::load(pa + i * kRowBytes, a[i]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) SmemVec<float, 2>::load(pb + j * kRowBytes, b[j]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
+            acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
+          }
+      }
+    }
+    team_barrier(team);                  // all four parts are done with the stage
+    if (issuer) {
+      fence_proxy_async();
+      issue(v + kQuadDepth);
+    }
+    since += 8;
+    if (since + 8 > kFlushCols) { flush<kQuadAcc>(acc, dacc, lane); since = 0; }
+  }
+  flush<kQuadAcc>(acc, dacc, lane);
+#pragma unroll
+  for (int k = 0; k < kQuadAcc / 32; ++k) totals[warp * kQuadAcc + lane * (kQuadAcc / 32) + k] = dacc[k];
+  __syncthreads();
+
+  // block totals: the two teams' sums of every part, in a fixed order
+  for (int idx = tid; idx < 4 * kQuadAcc; idx += kThreads) {
+    const int part = idx / kQuadAcc, e = idx - part * kQuadAcc;
+    int gi, gj;
+    if (part < 2) {
+      if (e >= 136) continue;
+      int i = 0, r = e;
+      while (r >= 16 - i) { r -= 16 - i; ++i; }
+      gi = 16 * part + i; gj = 16 * part + i + r;
+    } else {
+      if (e >= 128) continue;
+      gi = 8 * (part - 2) + e / 16; gj = 16 + e % 16;
+    }
+    if (gi >= prm.p || gj >= prm.p) continue;
+    const double sum = totals[(size_t)part * kQuadAcc + e] + totals[(size_t)(4 + part) * kQuadAcc + e];
+    prm.partials[(size_t)gram::canon_index(gi, gj, prm.p) * gridDim.x + blockIdx.x] = sum;
+  }
+  gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
+}
+
 namespace {
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -290,6 +428,35 @@ cudaError_t dispatch_tri(int pb, int vec, const Maps& maps, const Params& prm, c
 // few tiles per block, column coordinates within the 32-bit range of the copy instruction.
 bool gram_tm_eligible(const void* G, int dtype, int p, long long n) {
   return p >= 1 && p <= 16 && gramtm::available(G, dtype, n);
+}
+
+bool gram_tm32_eligible(const void* G, int dtype, int p, long long n) {
+  return dtype == 0 && p > 16 && p <= 32 && gramtm::available(G, dtype, n) && (n % 4) == 0;
+}
+
+cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
+                             int* status, cudaStream_t st) {
+  gramtm::Maps maps;
+  gramtm::Layout lay;
+  if (!gramtm::build(G, 0, p, n, maps, lay) || lay.q != 1) return cudaErrorInvalidValue;
+  gramtm::Params prm{};
+  prm.p = p;
+  prm.num_tiles = (n + gramtm::kTileCols - 1) / gramtm::kTileCols;
+  prm.partials = partials;
+  prm.counter = counter;
+  prm.K = K;
+  prm.status = status;
+  const int sms = sm_count();
+  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
+  cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
+  if (e != cudaSuccess) return e;
+  const size_t smem = (size_t)2 * gramtm::kQuadDepth * 32 * gramtm::kTileCols * 4 +
+                      (size_t)gramtm::kQuadWarps * gramtm::kQuadAcc * sizeof(double) +
+                      2 * gramtm::kQuadDepth * sizeof(uint64_t) + 64;
+  e = cudaFuncSetAttribute(gramtm::gram_quad_tm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  gramtm::gram_quad_tm_kernel<<<grid, gramtm::kQuadWarps * 32, smem, st>>>(maps, prm);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,

@@ -24,6 +24,11 @@ bool gram_tm_eligible(const void* G, int dtype, int p, long long n);
 cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
                            double* K, int* status, cudaStream_t st);
 
+// Tensor-fed Gram pass for fp32 with 16 < p <= 32 and rows on 16-byte boundaries.
+bool gram_tm32_eligible(const void* G, int dtype, int p, long long n);
+cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
+                             int* status, cudaStream_t st);
+
 // Persistent single-block IRLS on K (p x p).
 struct IrlsArgs {
   const double* K;

@@ -44,6 +44,9 @@ LADDER = [
     (64, 12_345, "gauss", False, 3),
     (5, 7, "gauss", True, 1), (15, 100_003, "noisy_mean", True, 0), (16, 50_000, "dup_zero", True, 4),
     (31, 40_002, "noisy_mean", True, 2), (63, 66_000, "dup_zero", True, 0), (64, 8_191, "gauss", True, 5),
+    # fp32, 16 < p <= 32, rows on 16-byte boundaries: the tensor-fed kernel with teams of four warps
+    (31, 50_000, "dup_zero", False, 0), (17, 4_096, "gauss", False, 0), (32, 300_004, "noisy_mean", False, 0),
+    (24, 1_000_000, "gauss", False, 4), (31, 4_100, "noisy_mean", False, 0),
     # bf16, p > 16, 16-byte aligned rows: the tensor-core kernel
     (17, 64, "gauss", True, 0), (33, 264, "noisy_mean", True, 0), (63, 4_096, "dup_zero", True, 0),
     (64, 65_536, "gauss", True, 0), (31, 1_000_000, "dup_zero", True, 8), (48, 300_008, "noisy_mean", True, 0),
@@ -286,6 +289,7 @@ AGG_LADDER = [
     (15, 65_537, "noisy_mean", False, 8, 0.01, 10, 1), (16, 70_000, "gauss", False, 8, 0.1, 6, 0),
     (17, 40_001, "noisy_mean", False, 9, 0.05, 6, 0), (31, 50_000, "dup_zero", False, 12, 0.01, 8, 2),
     (33, 20_000, "noisy_mean", False, 12, 0.0, 6, 0), (64, 12_345, "noisy_mean", False, 20, 0.01, 6, 3),
+    (31, 50_000, "dup_zero", False, 12, 0.01, 8, 0), (24, 1_000_000, "noisy_mean", False, 10, 0.02, 6, 4),
     (15, 100_003, "noisy_mean", True, 8, 0.01, 8, 0), (31, 40_002, "noisy_mean", True, 12, 0.02, 8, 2),
     (63, 66_000, "dup_zero", True, 16, 0.01, 8, 0), (33, 264, "noisy_mean", True, 10, 0.02, 6, 0),
     (64, 65_536, "noisy_mean", True, 20, 0.01, 6, 0), (31, 1_000_000, "dup_zero", True, 12, 0.01, 8, 8),
