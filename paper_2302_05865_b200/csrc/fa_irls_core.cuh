@@ -538,6 +538,19 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
       else {
         double acc = 0.0;
         for (int k = k0; k < r; ++k) { double v = Res[k * ld + i]; acc += v * v; }
+        if (a == 2.0 && cb == 1.0 && ca == 0.0) {
+          // the paper's square roots without a division or a square root: with y = 1/sqrt(acc fn),
+          // sqrt(u) = acc y and 1/(fn sqrt(u)) = y
+          const double fni = s.fn[i];
+          const double y = acc > 0.0 ? FA_RSQRT(acc * fni) : 0.0;
+          const double contrib = acc * y;
+          part += contrib;
+          wi = contrib >= kEps ? y : 1.0 / (fni * kEps);
+          ui = contrib * contrib;
+          s.u[i] = ui;
+          s.w[i] = wi;
+          continue;
+        }
         ui = acc / s.fn[i];
         double contrib, denom;
         term_of(ui, a, contrib, denom);
@@ -577,10 +590,17 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
         if (uniform) wij = coef;
         else {
           for (int k = k0; k < r; ++k) { double v = Res[k * ld + i] - Res[k * ld + j]; res2 += v * v; }
-          double contrib, denom;
-          term_of(res2 / d2, a, contrib, denom);
-          part += coef * contrib;
-          wij = coef / (d2 * denom);
+          if (a == 2.0) {
+            const double y = res2 > 0.0 ? FA_RSQRT(res2 * d2) : 0.0;     // sqrt(u) = res2 y, 1/(d2 sqrt(u)) = y
+            const double contrib = res2 * y;
+            part += coef * contrib;
+            wij = contrib >= kEps ? coef * y : coef / (d2 * kEps);
+          } else {
+            double contrib, denom;
+            term_of(res2 / d2, a, contrib, denom);
+            part += coef * contrib;
+            wij = coef / (d2 * denom);
+          }
         }
       }
       s.M[i * ld + j] = -2.0 * wij;
@@ -760,25 +780,28 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     int piv = -1;
     double dmax = kRankRel;
 #ifndef FA_IRLS_HOST
-    // every warp finds the pivot itself (two candidates per lane, butterfly); ties go to the lowest index
-    for (int j = (c.tid & 31); j < p; j += 32) {
-      const double dj = s.u[j];
-      if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
-    }
+    if (p > 32) {
+      // every warp finds the pivot itself (two candidates per lane, butterfly); ties go to the lowest index
+      for (int j = (c.tid & 31); j < p; j += 32) {
+        const double dj = s.u[j];
+        if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
+      }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const double od = __shfl_xor_sync(0xffffffffu, dmax, off);
-      const int oi = __shfl_xor_sync(0xffffffffu, piv, off);
-      if (od > dmax || (od == dmax && oi >= 0 && (piv < 0 || oi < piv))) { dmax = od; piv = oi; }
-    }
-#else
-    for (int j = 0; j < p; ++j) {                 // ties go to the lowest index
-      const double dj = s.u[j];
-      if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
-    }
+      for (int off = 16; off > 0; off >>= 1) {
+        const double od = __shfl_xor_sync(0xffffffffu, dmax, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, piv, off);
+        if (od > dmax || (od == dmax && oi >= 0 && (piv < 0 || oi < piv))) { dmax = od; piv = oi; }
+      }
+    } else
 #endif
+    {
+      for (int j = 0; j < p; ++j) {               // every thread scans; ties go to the lowest index
+        const double dj = s.u[j];
+        if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
+      }
+    }
     if (piv < 0) break;
-    const double rkk = sqrt(dmax), rinv = 1.0 / rkk;
+    const double rinv = FA_RSQRT(dmax), rkk = dmax * rinv;   // dmax in (1e-12, 1]: a normal number
     for (int j = c.tid; j < p; j += c.nt) {
       double v;
       if (j == piv) v = rkk;
