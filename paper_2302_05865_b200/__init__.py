@@ -21,7 +21,7 @@ ST_NONFINITE, ST_RANK0, ST_RANK_LT_M, ST_EIG_SWEEPS, ST_TIMEOUT = 1, 2, 4, 8, 16
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        f"{LIB_PATH} is missing: build it with `python -m paper_2302_05865_b200.build` "
+        f"{LIB_PATH} is missing: build it with `python paper_2302_05865_b200/build.py` "
         "(needs nvcc; there is no non-CUDA path)")
 _lib = ctypes.CDLL(LIB_PATH)
 
