@@ -198,6 +198,7 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
 constexpr int kQuadWarps = 8;
 constexpr int kQuadDepth = 3;                // stages per team: 2 x 3 x 32 KB
 constexpr int kQuadAcc = 160;                // 136 rounded up to a multiple of 32
+constexpr int kQuadFlushCols = 128;          // fp32 running sums cover at most this many columns here
 
 __device__ __forceinline__ void team_barrier(int team) {
   asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(128) : "memory");
@@ -226,18 +227,20 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   char* mystages = stages + (size_t)team * kQuadDepth * kStageBytes;
   uint64_t* mybars = full + team * kQuadDepth;
   const uint32_t tile_bytes = static_cast<uint32_t>(prm.p * kRowBytes);
-  // v-th tile of this team: the block's tile 2 v + team, i.e. global tile blockIdx.x + (2 v + team) * gridDim.x
-  auto tile_of = [&](long long v) { return (long long)blockIdx.x + (2 * v + team) * (long long)gridDim.x; };
-  auto issue = [&](long long v) {       // first lane of the team only
-    const long long t = tile_of(v);
-    if (t >= prm.num_tiles) return;
-    const int s = static_cast<int>(v % kQuadDepth);
+  // the team's tiles: global tiles blockIdx.x + (2 v + team) * gridDim.x, v = 0, 1, ...; tile numbers
+  // fit 32 bits (n < 2^31), and stage and phase are stepped along with the tile instead of being
+  // worked out from v (64-bit divisions by the depth were a visible part of the per-tile cost)
+  const int ntiles = static_cast<int>(prm.num_tiles);
+  const int tstride = 2 * static_cast<int>(gridDim.x);
+  const int tfirst = static_cast<int>(blockIdx.x) + team * static_cast<int>(gridDim.x);
+  auto issue = [&](int t, int s) {       // first lane of the team only
+    if (t >= ntiles) return;
     mbar_arrive_expect_tx(&mybars[s], tile_bytes);
-    tma_load_2d(mystages + (size_t)s * kStageBytes, &maps.map[0], static_cast<int>(t * kTileCols), 0, &mybars[s]);
+    tma_load_2d(mystages + (size_t)s * kStageBytes, &maps.map[0], t * kTileCols, 0, &mybars[s]);
   };
   const bool issuer = role == 0 && lane == 0;
   if (issuer)
-    for (int v = 0; v < kQuadDepth; ++v) issue(v);
+    for (int v = 0; v < kQuadDepth; ++v) issue(tfirst + v * tstride, v);
 
   float acc[kQuadAcc];
   double dacc[kQuadAcc / 32];
@@ -247,10 +250,10 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   for (int k = 0; k < kQuadAcc / 32; ++k) dacc[k] = 0.0;
   const int rowbase = (role < 2 ? 16 * role : 8 * (role - 2)) * kRowBytes;   // first row of the part (rectangle: its a-rows)
   int since = 0;
-  for (long long v = 0;; ++v) {
-    if (tile_of(v) >= prm.num_tiles) break;
-    const int s = static_cast<int>(v % kQuadDepth);
-    if (!mbar_wait(&mybars[s], static_cast<uint32_t>((v / kQuadDepth) & 1))) {
+  int s = 0;
+  uint32_t phase = 0;
+  for (int t = tfirst; t < ntiles; t += tstride) {
+    if (!mbar_wait(&mybars[s], phase)) {
       if (lane == 0 && prm.status) atomicOr(prm.status, kStTimeout);
       break;
     }
@@ -294,10 +297,11 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
     team_barrier(team);                  // all four parts are done with the stage
     if (issuer) {
       fence_proxy_async();
-      issue(v + kQuadDepth);
+      issue(t + kQuadDepth * tstride, s);
     }
+    if (++s == kQuadDepth) { s = 0; phase ^= 1u; }
     since += 8;
-    if (since + 8 > kFlushCols) { flush<kQuadAcc>(acc, dacc, lane); since = 0; }
+    if (since + 8 > kQuadFlushCols) { flush<kQuadAcc>(acc, dacc, lane); since = 0; }
   }
   flush<kQuadAcc>(acc, dacc, lane);
 #pragma unroll
