@@ -107,34 +107,39 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
   char* mystages = stages + (size_t)warp * depth * stage_bytes;
   uint64_t* mybars = full + warp * kMaxDepth;
 
-  // v-th tile of this warp: global tile blockIdx.x + (warp + v * 12) * gridDim.x, stage v mod depth
-  auto tile_of = [&](long long v) { return (long long)blockIdx.x + ((long long)warp + v * kTriWarps) * gridDim.x; };
-  auto issue = [&](long long v) {       // lane 0 only
-    const long long t = tile_of(v);
-    if (t >= prm.num_tiles) return;
-    const int s = static_cast<int>(v % depth);
+  // this warp's tiles: global tiles blockIdx.x + (warp + 12 v) * gridDim.x, v = 0, 1, ..., in stage
+  // v mod depth; tile numbers fit 32 bits, stage and phase are stepped along with the tile
+  const int ntiles = static_cast<int>(prm.num_tiles);
+  const int tstride = kTriWarps * static_cast<int>(gridDim.x);
+  const int tfirst = static_cast<int>(blockIdx.x) + warp * static_cast<int>(gridDim.x);
+  auto issue = [&](int t, int s) {       // lane 0 only
+    if (t >= ntiles) return;
     mbar_arrive_expect_tx(&mybars[s], static_cast<uint32_t>(stage_bytes));
     char* sbase = mystages + (size_t)s * stage_bytes;
-    const int x0 = static_cast<int>(t * lay.step);
+    const int x0 = t * lay.step;
     for (int cidx = 0; cidx < lay.q; ++cidx)
       if (lay.rows[cidx] > 0)
         tma_load_2d(sbase + (size_t)lay.rowbase[cidx] * kTileCols * S, &maps.map[cidx], x0, 0, &mybars[s]);
   };
   if (lane == 0)
-    for (int v = 0; v < depth; ++v) issue(v);
+    for (int v = 0; v < depth; ++v) issue(tfirst + v * tstride, v);
 
   const int groups = lay.step / V;
   const int per_tile = (groups + 31) / 32 * V;      // columns a thread takes from one tile
   int since = 0;
-  for (long long v = 0;; ++v) {
-    if (tile_of(v) >= prm.num_tiles) break;
-    const int s = static_cast<int>(v % depth);
-    if (!mbar_wait(&mybars[s], static_cast<uint32_t>((v / depth) & 1))) {
+  int s = 0;
+  uint32_t phase = 0;
+  for (int t = tfirst; t < ntiles; t += tstride) {
+    if (!mbar_wait(&mybars[s], phase)) {
       if (lane == 0) {
         if (prm.status) atomicOr(prm.status, kStTimeout);
         // let this warp's other loads land before the block can exit
-        for (long long w = v + 1; w < v + depth; ++w)
-          if (tile_of(w) < prm.num_tiles) (void)mbar_wait(&mybars[w % depth], static_cast<uint32_t>((w / depth) & 1));
+        int s2 = s;
+        uint32_t ph2 = phase;
+        for (int k = 1; k < depth; ++k) {
+          if (++s2 == depth) { s2 = 0; ph2 ^= 1u; }
+          if (t + k * tstride < ntiles) (void)mbar_wait(&mybars[s2], ph2);
+        }
       }
       break;
     }
@@ -162,8 +167,9 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
     __syncwarp();
     if (lane == 0) {
       fence_proxy_async();          // the warp's reads of this stage come before the next load's writes
-      issue(v + depth);
+      issue(t + depth * tstride, s);
     }
+    if (++s == depth) { s = 0; phase ^= 1u; }
     since += per_tile;
     if (since + per_tile > kFlushCols) { flush<NACCP>(acc, dacc, lane); since = 0; }
   }
