@@ -284,8 +284,8 @@ def main():
 
     peak, peak_src = measured_peaks()
     # DRAM bytes per Gram launch from the ncu capture summarised in profiles/gram_tri_tm_f32_p15_cfg2.md
-    # (250.7 MB at n = 4,000,000, scaled by n); only valid for that kernel and workload
-    traffic = int(250.74e6 * w.n / 4_000_000) if (w.p == 15 and w.dtype == "f32" and w.n >= 4096) else None
+    # (252.2 MB at n = 4,000,000, scaled by n); only valid for that kernel and workload
+    traffic = int(252.16e6 * w.n / 4_000_000) if (w.p == 15 and w.dtype == "f32" and w.n >= 4096) else None
     gram_bytes = w.p * w.n * w.itemsize
     comb_bytes = w.p * w.n * w.itemsize + 4 * w.n
     gram_gbs = gram_bytes / (t_gram * 1e-3) / 1e9

@@ -1,16 +1,21 @@
 // Gram pass on the 5th-generation tensor cores, for bf16 gradients with 16 < p <= 64 workers
 // (K = G G^T needs 16 FMA per byte at p = 63, far beyond the fp32 pipes at HBM speed).
 //
-// One persistent block per SM, three roles:
+// One persistent block per SM, four roles:
 //   warp 0   : TMA producer.  The gradient matrix is a 2-D tensor (n columns x p rows, row stride n);
 //              a box of 64 columns x 64 rows (rows >= p and columns >= n read as zero) lands in
-//              shared memory in the 128-byte-swizzled K-major layout the MMA unit reads.
+//              shared memory in the 128-byte-swizzled K-major layout the MMA unit reads.  The
+//              tensor-load unit delivers about 14 bytes per clock and SM for such 128-byte rows,
+//              less than HBM supplies, so it fills four of the six stages only.
+//   warps 6-9: loaders.  The other two stages (every third tile) are filled with 16-byte cp.async
+//              copies written straight into the same swizzled layout, two tiles in flight.
 //   warp 1   : MMA issuer.  One thread issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with the
 //              SAME shared-memory tile as A and B operand: D[64 x 64] += T T^T, 16 columns per
-//              instruction, accumulator in tensor memory.  tcgen05.commit frees the stage.
-//   warps 2-5: epilogue.  After every stage (256 columns) the fp32 accumulator (products are exact, the
-//              running sum is fp32) is read out of tensor memory with tcgen05.ld and added into
-//              fp64 registers; two accumulators alternate so the MMAs never wait for the read-out.
+//              instruction, accumulator in tensor memory (eight accumulators used in turn).
+//              tcgen05.commit frees the stage.
+//   warps 2-5: read-out.  After every stage (256 columns) the fp32 accumulator (products are exact,
+//              the running sum is fp32) is read out of tensor memory with tcgen05.ld and added into
+//              fp32 registers; every eighth run these are folded into fp64 sums in shared memory.
 // Block totals then go through the same last-block reduction as the fp32-pipe kernels.
 // Needs 16-byte aligned rows (n % 8 == 0, base % 16 == 0); other shapes use the fp32-pipe kernel.
 #include <cuda.h>
@@ -30,12 +35,37 @@ constexpr int kBoxesPerStage = 4;               // 256 columns per stage
 constexpr int kStageBytes = kBoxBytes * kBoxesPerStage;
 constexpr int kStages = 6;                      // 192 KiB of staging
 constexpr int kFlushStages = 1;                 // 256 columns per fp32 accumulation run
-constexpr int kThreads = 192;
-constexpr int kTmemCols = 128;                  // two 64-column accumulators
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+constexpr int kFold = 8;                        // runs added in fp32 registers before the fp64 fold
+constexpr int kLoaderWarps = 4;                 // warps 6..9 fill every third stage with plain loads
+constexpr int kThreads = 192 + 32 * kLoaderWarps;
+#ifndef FA_TC_ACCS
+#define FA_TC_ACCS 8
+#endif
+constexpr int kAccs = FA_TC_ACCS;               // 64-column accumulators in tensor memory, used in turn
+constexpr int kTmemCols = 64 * kAccs;
+static_assert(kAccs == 2 || kAccs == 4 || kAccs == 8, "tensor-memory allocations are powers of two");
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 64 * 64 * sizeof(double);
+
+// Stages whose bit is set in kLoaderMask are filled by the loader warps, the others by the
+// tensor-load thread; tile u goes to stage u mod kStages.
+#ifndef FA_TC_LOADER_MASK
+#define FA_TC_LOADER_MASK 0x24
+#endif
+constexpr uint32_t kLoaderMask = FA_TC_LOADER_MASK;
+constexpr int kLoaderDepth = ((kLoaderMask >> 0) & 1) + ((kLoaderMask >> 1) & 1) + ((kLoaderMask >> 2) & 1) +
+                             ((kLoaderMask >> 3) & 1) + ((kLoaderMask >> 4) & 1) + ((kLoaderMask >> 5) & 1);
+static_assert(kLoaderDepth >= 1 && kLoaderDepth <= 3 && kLoaderMask < (1u << kStages), "loader stages");
+__device__ __forceinline__ bool loader_stage(int s) { return (kLoaderMask >> s) & 1u; }
+__device__ __forceinline__ bool loader_tile(long long u) { return loader_stage(static_cast<int>(u % kStages)); }
+__device__ __forceinline__ long long next_loader_tile(long long u) {
+  do { ++u; } while (!loader_tile(u));
+  return u;
+}
 
 struct Params {
   int p;
+  const uint4* G;            // the matrix as 16-byte chunks (rows start on 16-byte boundaries)
+  long long n;
   long long num_tiles;       // stages' worth of columns in the whole matrix
   double* partials;
   unsigned int* counter;
@@ -93,8 +123,8 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 struct Bars {
   uint64_t full[kStages];
   uint64_t empty[kStages];
-  uint64_t acc_full[2];
-  uint64_t acc_empty[2];
+  uint64_t acc_full[kAccs];
+  uint64_t acc_empty[kAccs];
   uint32_t tmem_base;
   int abort;
 };
@@ -110,19 +140,32 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
   unsigned char* stages =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   Bars* bars = reinterpret_cast<Bars*>(stages + (size_t)kStages * kStageBytes);
+  double* dsum = reinterpret_cast<double*>(stages + (size_t)kStages * kStageBytes + 256);   // 64 x 64 fp64 sums
+  static_assert(sizeof(Bars) <= 256, "barrier block");
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 4); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&bars->full[s], loader_stage(s) ? kLoaderWarps : 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    for (int a = 0; a < kAccs; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 4); }
     bars->abort = 0;
     fence_proxy_async();
   }
-  if (warp == 1) {   // tensor memory: 128 columns for this block (the only block on the SM)
+  if (warp == 1) {   // tensor memory: kTmemCols columns for this block (the only block on the SM)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int i = tid; i < 64 * 64; i += kThreads) dsum[i] = 0.0;
+  if (warp >= 6) {   // rows p..63 of the stages the loader warps fill are zeroed once and never written
+    for (int s = 0; s < kStages; ++s)
+      if (loader_stage(s))
+      for (int i = (tid - 192) * 16; i < kStageBytes; i += 32 * kLoaderWarps * 16)
+        *reinterpret_cast<uint4*>(stages + (size_t)s * kStageBytes + i) = make_uint4(0, 0, 0, 0);
+    fence_proxy_async();
   }
   tc_fence_before();
   __syncthreads();
@@ -139,6 +182,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
       long long issued = 0;
       bool ok = true;
       for (long long u = 0; u < my_tiles; ++u) {
+        if (loader_tile(u)) continue;
         const int s = static_cast<int>(u % kStages);
         if (!mbar_wait(&bars->empty[s], static_cast<uint32_t>(((u / kStages) & 1) ^ 1)) ||
             *reinterpret_cast<volatile int*>(&bars->abort)) { ok = false; break; }
@@ -153,7 +197,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
         give_up(bars, prm.status);
         const long long first = issued > kStages ? issued - kStages : 0;   // copies still in flight must land
         for (long long u = first; u < issued; ++u)
-          (void)mbar_wait(&bars->full[u % kStages], static_cast<uint32_t>((u / kStages) & 1));
+          if (!loader_tile(u)) (void)mbar_wait(&bars->full[u % kStages], static_cast<uint32_t>((u / kStages) & 1));
       }
     }
   } else if (warp == 1) {
@@ -162,10 +206,10 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
       for (long long u = 0; u < my_tiles; ++u) {
         const int s = static_cast<int>(u % kStages);
         const long long period = u / kFlushStages;
-        const int ab = static_cast<int>(period & 1);
+        const int ab = static_cast<int>(period % kAccs);
         const bool first_of_period = (u % kFlushStages) == 0;
-        if (first_of_period && period >= 2) {     // the epilogue must have drained this accumulator
-          if (!mbar_wait(&bars->acc_empty[ab], static_cast<uint32_t>(((period >> 1) - 1) & 1))) { give_up(bars, prm.status); break; }
+        if (first_of_period && period >= kAccs) {     // the epilogue must have drained this accumulator
+          if (!mbar_wait(&bars->acc_empty[ab], static_cast<uint32_t>(((period / kAccs) - 1) & 1))) { give_up(bars, prm.status); break; }
         }
         if (!mbar_wait(&bars->full[s], static_cast<uint32_t>((u / kStages) & 1))) { give_up(bars, prm.status); break; }
         if (*reinterpret_cast<volatile int*>(&bars->abort)) break;
@@ -184,18 +228,97 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
         if ((u % kFlushStages) == kFlushStages - 1 || u == my_tiles - 1) umma_commit(&bars->acc_full[ab]);
       }
     }
+  } else if (warp >= 6) {
+    // ---------------- loader warps: the tensor-load unit delivers about 14 bytes per clock for boxes
+    // with 128-byte rows, well below what HBM can supply, so every third tile comes in through the
+    // load/store path instead: 16-byte asynchronous copies (cp.async; a warp covers the 512 contiguous
+    // bytes of one row of the tile) straight into the layout the 128-byte swizzled tensor load would
+    // have produced -- box q = 64 columns, row r at r * 128 bytes, 16-byte chunk c at position
+    // c ^ (r mod 8).  Two tiles are in flight (one per loader stage); a tile is handed to the tensor
+    // core once every thread's copies have landed and a proxy fence has made them visible to it.
+    const int lt = tid - 192;
+    const int chunks = prm.p * 32;                        // 16-byte chunks of a tile: p rows x 512 bytes
+    const long long row_chunks = prm.n / 8;
+    constexpr int kPer = 2048 / (32 * kLoaderWarps);      // chunks per thread and tile
+    bool ok = true;
+    auto fill = [&](long long u) {                        // wait for the stage of tile u, start its copies
+      const int s = static_cast<int>(u % kStages);
+      ok = mbar_wait(&bars->empty[s], static_cast<uint32_t>(((u / kStages) & 1) ^ 1)) &&
+           !*reinterpret_cast<volatile int*>(&bars->abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) return;
+      const long long t = blockIdx.x + u * (long long)gridDim.x;
+      const long long chunk0 = t * (kBoxesPerStage * kBoxCols / 8);   // first chunk of the tile within a row
+      const uint32_t sbase = smem_u32(stages + (size_t)s * kStageBytes);
+#pragma unroll
+      for (int k = 0; k < kPer; ++k) {
+        const int idx = lt + k * 32 * kLoaderWarps;
+        const int r = idx >> 5, ch = idx & 31;
+        if (idx < chunks) {
+          const bool inside = chunk0 + ch < row_chunks;   // chunks past the end of the row are zero-filled
+          const uint4* src = inside ? prm.G + (size_t)r * row_chunks + chunk0 + ch : prm.G;
+          const uint32_t dst = sbase + (ch >> 3) * kBoxBytes + r * 128 + (((ch & 7) ^ (r & 7)) << 4);
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(inside ? 16 : 0)
+                       : "memory");
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // loader tiles in order; `head` is the next one to start, `tail` the next one to hand over;
+    // kLoaderDepth of them (one per loader stage) are in flight
+    long long head = next_loader_tile(-1), tail = head;
+    for (int i = 0; i < kLoaderDepth - 1 && head < my_tiles && ok; ++i) {
+      fill(head);
+      head = next_loader_tile(head);
+    }
+    while (tail < my_tiles && ok) {
+      const bool more = head < my_tiles;
+      if (more) {
+        fill(head);
+        head = next_loader_tile(head);
+        if (!ok) break;
+      }
+      // copy groups complete in order: with kLoaderDepth groups committed the oldest has landed when
+      // at most kLoaderDepth - 1 are pending; near the end simply wait for all of them
+      if (more && kLoaderDepth == 3) asm volatile("cp.async.wait_group 2;" ::: "memory");
+      else if (more && kLoaderDepth == 2) asm volatile("cp.async.wait_group 1;" ::: "memory");
+      else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      fence_proxy_async();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->full[static_cast<int>(tail % kStages)]);
+      tail = next_loader_tile(tail);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");   // nothing of this thread's is in flight at exit
+    if (!ok && lane == 0) give_up(bars, prm.status);
   } else {
     // ---------------- epilogue: warp w reads TMEM lanes 32*(w%4) .. +31; with M = 64 only the first
     // 16 lanes of each quarter carry rows: row = 16*(w%4) + lane
     const int quarter = warp & 3;
     const int row = 16 * quarter + (lane & 15);
-    double dacc[64];
+    // Read-out per 256-column run: the fp32 values are added into fp32 registers (round to nearest;
+    // kFold runs), and only every kFold-th run are these folded into the fp64 sums, which live in
+    // shared memory (entry (row, j) at j * 64 + row: the rows of a warp are neighbours).  Converting
+    // and adding all 64 values in fp64 after every run made the read-out the slowest stage of the
+    // pipeline (2300 cycles per run).
+    float facc[64];
 #pragma unroll
-    for (int j = 0; j < 64; ++j) dacc[j] = 0.0;
+    for (int j = 0; j < 64; ++j) facc[j] = 0.f;
+    int in_fold = 0;
+    bool first_fold = true;
+    auto fold = [&]() {
+      if (lane < 16) {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) dsum[j * 64 + row] += static_cast<double>(facc[j]);
+      }
+#pragma unroll
+      for (int j = 0; j < 64; ++j) facc[j] = 0.f;
+      first_fold = false;
+      in_fold = 0;
+    };
     bool ok = true;
     for (long long period = 0; period < periods && ok; ++period) {
-      const int ab = static_cast<int>(period & 1);
-      if (!mbar_wait(&bars->acc_full[ab], static_cast<uint32_t>((period >> 1) & 1))) {
+      const int ab = static_cast<int>(period % kAccs);
+      if (!mbar_wait(&bars->acc_full[ab], static_cast<uint32_t>((period / kAccs) & 1))) {
         if (lane == 0) give_up(bars, prm.status);
         ok = false;
         break;
@@ -211,13 +334,15 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
       if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
-        dacc[j] += static_cast<double>(__uint_as_float(v0[j]));
-        dacc[32 + j] += static_cast<double>(__uint_as_float(v1[j]));
+        facc[j] += __uint_as_float(v0[j]);
+        facc[32 + j] += __uint_as_float(v1[j]);
       }
+      if (++in_fold == kFold) fold();
     }
+    if (in_fold > 0 || first_fold) fold();
     if (lane < 16 && row < prm.p) {
       for (int j = row; j < prm.p; ++j)
-        prm.partials[(size_t)gram::canon_index(row, j, prm.p) * gridDim.x + blockIdx.x] = dacc[j];
+        prm.partials[(size_t)gram::canon_index(row, j, prm.p) * gridDim.x + blockIdx.x] = dsum[j * 64 + row];
     }
   }
 
@@ -276,6 +401,8 @@ cudaError_t launch_gram_tc(const void* G, int p, long long n, double* partials, 
     return cudaErrorInvalidValue;
   gramtc::Params prm{};
   prm.p = p;
+  prm.G = static_cast<const uint4*>(G);
+  prm.n = n;
   const long long stage_cols = gramtc::kBoxesPerStage * gramtc::kBoxCols;
   prm.num_tiles = (n + stage_cols - 1) / stage_cols;
   prm.partials = partials;
