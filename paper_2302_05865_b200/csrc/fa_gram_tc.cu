@@ -37,7 +37,8 @@ constexpr int kStages = 6;                      // 192 KiB of staging
 constexpr int kFlushStages = 1;                 // 256 columns per fp32 accumulation run
 constexpr int kFold = 8;                        // runs added in fp32 registers before the fp64 fold
 constexpr int kLoaderWarps = 4;                 // warps 6..9 fill every third stage with plain loads
-constexpr int kThreads = 192 + 32 * kLoaderWarps;
+constexpr int kMmaWarp2 = 6 + kLoaderWarps;       // second MMA issuer (odd tiles); warp 1 takes the even ones
+constexpr int kThreads = 192 + 32 * kLoaderWarps + 32;
 #ifndef FA_TC_ACCS
 #define FA_TC_ACCS 8
 #endif
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   for (int i = tid; i < 64 * 64; i += kThreads) dsum[i] = 0.0;
-  if (warp >= 6) {   // rows p..63 of the stages the loader warps fill are zeroed once and never written
+  if (warp >= 6 && warp < 6 + kLoaderWarps) {   // rows p..63 of the stages the loader warps fill are zeroed once and never written
     for (int s = 0; s < kStages; ++s)
       if (loader_stage(s))
       for (int i = (tid - 192) * 16; i < kStageBytes; i += 32 * kLoaderWarps * 16)
@@ -200,10 +201,12 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
           if (!loader_tile(u)) (void)mbar_wait(&bars->full[u % kStages], static_cast<uint32_t>((u / kStages) & 1));
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer
+  } else if (warp == 1 || warp == kMmaWarp2) {
+    // ---------------- MMA issuers: one thread each, tiles of one parity (its own accumulators: tile u
+    // uses accumulator u mod kAccs, and kAccs is even); a commit covers the issuing thread's MMAs
+    static_assert(kFlushStages == 1 && kAccs % 2 == 0, "tiles alternate between the two issuers");
     if (lane == 0) {
-      for (long long u = 0; u < my_tiles; ++u) {
+      for (long long u = (warp == 1 ? 0 : 1); u < my_tiles; u += 2) {
         const int s = static_cast<int>(u % kStages);
         const long long period = u / kFlushStages;
         const int ab = static_cast<int>(period % kAccs);
@@ -228,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
         if ((u % kFlushStages) == kFlushStages - 1 || u == my_tiles - 1) umma_commit(&bars->acc_full[ab]);
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 6 && warp < 6 + kLoaderWarps) {
     // ---------------- loader warps: the tensor-load unit delivers about 14 bytes per clock for boxes
     // with 128-byte rows, well below what HBM can supply, so every third tile comes in through the
     // load/store path instead: 16-byte asynchronous copies (cp.async; a warp covers the 512 contiguous
@@ -290,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");   // nothing of this thread's is in flight at exit
     if (!ok && lane == 0) give_up(bars, prm.status);
-  } else {
+  } else if (warp < 6) {
     // ---------------- epilogue: warp w reads TMEM lanes 32*(w%4) .. +31; with M = 64 only the first
     // 16 lanes of each quarter carry rows: row = 16*(w%4) + lane
     const int quarter = warp & 3;
