@@ -1,7 +1,7 @@
 // Gram pass on the 5th-generation tensor cores, for bf16 gradients with 16 < p <= 64 workers
 // (K = G G^T needs 16 FMA per byte at p = 63, far beyond the fp32 pipes at HBM speed).
 //
-// One persistent block per SM, four roles:
+// One persistent block per SM (352 threads), four roles:
 //   warp 0   : TMA producer.  The gradient matrix is a 2-D tensor (n columns x p rows, row stride n);
 //              a box of 64 columns x 64 rows (rows >= p and columns >= n read as zero) lands in
 //              shared memory in the 128-byte-swizzled K-major layout the MMA unit reads.  The
@@ -9,10 +9,11 @@
 //              less than HBM supplies, so it fills four of the six stages only.
 //   warps 6-9: loaders.  The other two stages (every third tile) are filled with 16-byte cp.async
 //              copies written straight into the same swizzled layout, two tiles in flight.
-//   warp 1   : MMA issuer.  One thread issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32) with the
-//              SAME shared-memory tile as A and B operand: D[64 x 64] += T T^T, 16 columns per
-//              instruction, accumulator in tensor memory (eight accumulators used in turn).
-//              tcgen05.commit frees the stage.
+//   warps 1, 10: MMA issuers.  One thread each issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32)
+//              with the SAME shared-memory tile as A and B operand: D[64 x 64] += T T^T, 16 columns
+//              per instruction, accumulator in tensor memory (eight accumulators used in turn).
+//              Warp 1 takes the even tiles, warp 10 the odd ones: sixteen small instructions per
+//              tile from one thread were slower than the feed.  tcgen05.commit frees the stage.
 //   warps 2-5: read-out.  After every stage (256 columns) the fp32 accumulator (products are exact,
 //              the running sum is fp32) is read out of tensor memory with tcgen05.ld and added into
 //              fp32 registers; every eighth run these are folded into fp64 sums in shared memory.
