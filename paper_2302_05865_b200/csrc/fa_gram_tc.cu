@@ -6,9 +6,9 @@
 //              a box of 64 columns x 64 rows (rows >= p and columns >= n read as zero) lands in
 //              shared memory in the 128-byte-swizzled K-major layout the MMA unit reads.  The
 //              tensor-load unit delivers about 14 bytes per clock and SM for such 128-byte rows,
-//              less than HBM supplies, so it fills four of the six stages only.
-//   warps 6-9: loaders.  The other two stages (every third tile) are filled with 16-byte cp.async
-//              copies written straight into the same swizzled layout, two tiles in flight.
+//              less than HBM supplies, so it fills three of the six stages only (the even tiles).
+//   warps 6-9: loaders.  The other three stages (the odd tiles) are filled with 16-byte cp.async
+//              copies written straight into the same swizzled layout, three tiles in flight.
 //   warps 1, 10: MMA issuers.  One thread each issues tcgen05.mma (kind::f16, bf16 x bf16 -> fp32)
 //              with the SAME shared-memory tile as A and B operand: D[64 x 64] += T T^T, 16 columns
 //              per instruction, accumulator in tensor memory (eight accumulators used in turn).
@@ -37,7 +37,7 @@ constexpr int kStageBytes = kBoxBytes * kBoxesPerStage;
 constexpr int kStages = 6;                      // 192 KiB of staging
 constexpr int kFlushStages = 1;                 // 256 columns per fp32 accumulation run
 constexpr int kFold = 8;                        // runs added in fp32 registers before the fp64 fold
-constexpr int kLoaderWarps = 4;                 // warps 6..9 fill every third stage with plain loads
+constexpr int kLoaderWarps = 4;                 // warps 6..9 fill the loader stages with cp.async copies
 constexpr int kMmaWarp2 = 6 + kLoaderWarps;       // second MMA issuer (odd tiles); warp 1 takes the even ones
 constexpr int kThreads = 192 + 32 * kLoaderWarps + 32;
 #ifndef FA_TC_ACCS
@@ -51,7 +51,7 @@ constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 64 * 
 // Stages whose bit is set in kLoaderMask are filled by the loader warps, the others by the
 // tensor-load thread; tile u goes to stage u mod kStages.
 #ifndef FA_TC_LOADER_MASK
-#define FA_TC_LOADER_MASK 0x24
+#define FA_TC_LOADER_MASK 0x2A
 #endif
 constexpr uint32_t kLoaderMask = FA_TC_LOADER_MASK;
 constexpr int kLoaderDepth = ((kLoaderMask >> 0) & 1) + ((kLoaderMask >> 1) & 1) + ((kLoaderMask >> 2) & 1) +
@@ -234,11 +234,11 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
     }
   } else if (warp >= 6 && warp < 6 + kLoaderWarps) {
     // ---------------- loader warps: the tensor-load unit delivers about 14 bytes per clock for boxes
-    // with 128-byte rows, well below what HBM can supply, so every third tile comes in through the
+    // with 128-byte rows, well below what HBM can supply, so every other tile comes in through the
     // load/store path instead: 16-byte asynchronous copies (cp.async; a warp covers the 512 contiguous
     // bytes of one row of the tile) straight into the layout the 128-byte swizzled tensor load would
     // have produced -- box q = 64 columns, row r at r * 128 bytes, 16-byte chunk c at position
-    // c ^ (r mod 8).  Two tiles are in flight (one per loader stage); a tile is handed to the tensor
+    // c ^ (r mod 8).  As many tiles are in flight as there are loader stages; a tile is handed to the tensor
     // core once every thread's copies have landed and a proxy fence has made them visible to it.
     const int lt = tid - 192;
     const int chunks = prm.p * 32;                        // 16-byte chunks of a tile: p rows x 512 bytes
