@@ -42,6 +42,11 @@ each other: "literal" builds the n x n matrix C term by term (small n only);
 "svd" uses C = B B^T with B = G^T M^(1/2), M = diag(w) + sum w_ij (e_i-e_j)
 (e_i-e_j)^T, and takes the left singular vectors of the n x p matrix B.
 
+fa_aggregate_blocked is the "svd" iteration for gradient lengths whose fp64
+copies do not fit in memory: the same rounds with every n-vector visited in
+column blocks (the thin SVD of B through the triangular factor of a QR that
+takes B one block of rows at a time).  It is pinned against fa_aggregate.
+
 Parity pins (tests/test_oracle_pins.py): mean recovery, orthonormality and
 ratio range, PCA special case, worker-permutation and scaling invariance,
 monotone descent, first-order stationarity of Eq. (5) at the fixed point by
@@ -77,12 +82,6 @@ def pair_sqdist(G: np.ndarray) -> np.ndarray:
             diff = G[i] - G[j]
             D2[i, j] = D2[j, i] = float(diff @ diff)
     return D2
-
-
-def residual_ratio(Y: np.ndarray, x: np.ndarray) -> float:
-    """1 - ||Y^T x||^2/||x||^2 written as ||x - Y Y^T x||^2 / ||x||^2."""
-    res = x - Y @ (Y.T @ x)
-    return float(res @ res) / float(x @ x)
 
 
 def _classify(G):
@@ -328,6 +327,156 @@ def fa_aggregate(G, m, lam=0.0, iters=5, method="svd", eps=EPS, history=False, a
             break
     d = Y @ (Y.T @ G.sum(axis=0)) / p
     return dict(d=d, Y=Y, u=u, w=w, objective=objs, rounds=len(objs), evals=evals, Ys=Ys)
+
+
+# -- the same iteration for any n: every n-vector is visited in column blocks ----------------
+
+def _blocks(n, block):
+    return [(c0, min(c0 + block, n)) for c0 in range(0, n, block)]
+
+
+def _for_blocks(fn, spans, threads):
+    """fn(c0, c1) for every column block, results in block order (plain loop unless threads > 1)."""
+    if threads <= 1:
+        return [fn(c0, c1) for c0, c1 in spans]
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(threads) as ex:
+        return list(ex.map(lambda s: fn(*s), spans))
+
+
+def fa_aggregate_blocked(G, m, lam=0.0, iters=5, block=1 << 16, widen=None, eps=EPS, sample=None, threads=1):
+    """fa_aggregate(..., method="svd") with a = 2 and the Beta(1, 1/2) likelihood of Eq. (1), for any n.
+
+    The rounds, weights, term values and the final average are those of fa_aggregate; what changes
+    is only how the n-dimensional objects are held.  G stays in its storage type and is widened
+    to fp64 one column block at a time (`widen`, default: plain conversion), and Y (n x m) is never
+    kept: per round
+      1. the thin SVD of B = G^T M^(1/2) (n x p) is taken through a QR that sees B one block of
+         rows at a time (R of [R_so_far; B_block]), then R = U S V^T, so that B = (Q U) S V^T and the
+         left singular vectors are Y = B V S^-1, formed block by block;
+      2. Z = G Y (p x k: the coordinates Y^T g_i of every gradient) is summed over the blocks;
+      3. the residual rows r_i = g_i - Y Y^T g_i are formed block by block and their squared norms,
+         and those of the explicit differences r_i - r_j of the active pairs, are summed.
+    After the last round d = (1/p) Y (Y^T G 1) is formed block by block.
+
+    sample  : optional integer array of column indices; d is then returned only there (d_sample),
+              together with its full norm (d_norm), instead of as a full vector
+    threads : column blocks of one pass may be worked on by this many threads (sums are still added
+              in block order)
+    returns : dict with objective (one per round), u, w, evals (last round), k, Z = G Y (p x k) of the
+              last round, yty_err = max |Y^T Y - I| of the last round, K = G G^T, D2, d or
+              (d_sample, d_norm).
+    """
+    p, n = G.shape
+    if widen is None:
+        widen = lambda x: np.asarray(x, dtype=np.float64)
+    if not (1 <= m <= p) or iters < 1 or lam < 0:
+        raise ValueError("need 1 <= m <= p, iters >= 1, lam >= 0")
+    spans = _blocks(n, int(block))
+    coef = lam / (p - 1) if (lam > 0 and p > 1) else 0.0
+
+    # inner products, and D_ij^2 from the difference vectors
+    def first_pass(c0, c1):
+        X = widen(G[:, c0:c1])
+        return X @ X.T, (pair_sqdist(X) if coef > 0 else None)
+    K = np.zeros((p, p))
+    D2 = np.zeros((p, p))
+    for Kb, Db in _for_blocks(first_pass, spans, threads):
+        K += Kb
+        if Db is not None:
+            D2 += Db
+    norms = np.diag(K).copy()
+    zero = norms <= ZERO_NORM_REL * float(norms.max())
+    active = np.zeros((p, p), dtype=bool)
+    if coef > 0:
+        active = D2 > SAME_PAIR_REL * (norms[:, None] + norms[None, :])
+        np.fill_diagonal(active, False)
+    if np.all(zero):
+        out = dict(objective=[0.0] * iters, u=np.zeros(p), w=np.zeros(p), evals=np.zeros(p), k=0,
+                   Z=np.zeros((p, 0)), yty_err=0.0, K=K, D2=D2)
+        if sample is None:
+            out["d"] = np.zeros(n)
+        else:
+            out["d_sample"], out["d_norm"] = np.zeros(len(sample)), 0.0
+        return out
+
+    u = np.zeros(p)
+    U = np.zeros((p, p))
+    objs = []
+    for t in range(1, iters + 1):
+        w = np.zeros(p)
+        W = np.zeros((p, p))
+        if t == 1:
+            w[~zero] = 1.0
+            W[active] = coef
+        else:
+            w[~zero] = 1.0 / (norms[~zero] * np.maximum(np.sqrt(np.maximum(u[~zero], 0.0)), eps))
+            if coef > 0:
+                W[active] = coef / (D2[active] * np.maximum(np.sqrt(np.maximum(U[active], 0.0)), eps))
+        # M^(1/2) as in weighted_pca_svd
+        if np.any(W != 0.0):
+            e, E = np.linalg.eigh(pair_weight_matrix(w, W))
+            S = E * np.sqrt(np.maximum(e, 0.0))[None, :]
+        else:
+            S = np.diag(np.sqrt(w))
+        # 1. triangular factor of B, one block of rows at a time
+        Rfac = np.zeros((0, p))
+        for B in _for_blocks(lambda c0, c1: np.linalg.qr(widen(G[:, c0:c1]).T @ S, mode="r"), spans, threads):
+            Rfac = np.linalg.qr(np.vstack([Rfac, B]), mode="r")
+        _, sv, Vt = np.linalg.svd(Rfac)
+        evals = sv * sv
+        k = _keep(evals, min(m, n))
+        Ymap = S @ (Vt[:k].T / sv[:k][None, :])          # Y_block = G_block^T Ymap  (= B_block V S^-1)
+        # 2. coordinates of every gradient, and Y^T Y as a check on the blocked SVD
+        def second_pass(c0, c1):
+            X = widen(G[:, c0:c1])
+            Yb = X.T @ Ymap
+            return X @ Yb, Yb.T @ Yb
+        Z = np.zeros((p, k))
+        YtY = np.zeros((k, k))
+        for Zb, Yb2 in _for_blocks(second_pass, spans, threads):
+            Z += Zb
+            YtY += Yb2
+        # 3. residual rows and the values under the roots of Eq. (5)
+        def third_pass(c0, c1):
+            X = widen(G[:, c0:c1])
+            R = X - Z @ (X.T @ Ymap).T
+            return np.einsum("ij,ij->i", R, R), (pair_sqdist(R) if coef > 0 else None)
+        rr = np.zeros(p)
+        RR = np.zeros((p, p))
+        for rb, Rb in _for_blocks(third_pass, spans, threads):
+            rr += rb
+            if Rb is not None:
+                RR += Rb
+        u = np.zeros(p)
+        u[~zero] = rr[~zero] / norms[~zero]
+        U = np.zeros((p, p))
+        U[active] = RR[active] / D2[active]
+        obj = float(np.sum(np.sqrt(np.maximum(u, 0.0))))
+        if coef > 0:
+            obj += coef * float(np.sum(np.sqrt(np.maximum(U, 0.0))))
+        objs.append(obj)
+
+    # d = (1/p) Y (Y^T sum_i g_i); Y^T sum_i g_i = sum_i Z[i]
+    zsum = Z.sum(axis=0) / p
+    out = dict(objective=objs, u=u, w=w, evals=evals, k=k, Z=Z, K=K, D2=D2,
+               yty_err=float(np.abs(YtY - np.eye(k)).max()) if k else 0.0)
+    if sample is None:
+        d = np.empty(n)
+        for c0, c1 in spans:
+            d[c0:c1] = (widen(G[:, c0:c1]).T @ Ymap) @ zsum
+        out["d"] = d
+    else:
+        sample = np.asarray(sample, dtype=np.int64)
+        d_sample = np.empty(sample.size)
+        norm2 = 0.0
+        for c0, c1 in spans:
+            db = (widen(G[:, c0:c1]).T @ Ymap) @ zsum
+            norm2 += float(db @ db)
+            sel = (sample >= c0) & (sample < c1)
+            d_sample[sel] = db[sample[sel] - c0]
+        out["d_sample"], out["d_norm"] = d_sample, float(np.sqrt(norm2))
+    return out
 
 
 def reconstruction(G, Y):

@@ -51,6 +51,37 @@ def test_workspace_query_and_error_codes_without_a_device(lib):
     assert lib.fa_aggregate(None, 0, 4, 10, 2, 0.0, 3, None, None, None, 0, None, None) == -1
 
 
+def test_binding_rejects_wrong_buffers_before_any_launch(lib):
+    """Every tensor handed to the binding is checked for element type and size on the host: a float32
+    A_out or an obj_out shorter than `iters` would otherwise be an out-of-bounds write on the device.
+    (Checked in this order: type, contiguity, size, device -- so CPU tensors reach the first three.)"""
+    import torch
+    import paper_2302_05865_b200 as fa
+    ok = torch.zeros(15 * 8, dtype=torch.float64)
+    for bad, what in ((torch.zeros(15 * 8, dtype=torch.float32), "dtype"), (torch.zeros(15 * 8 - 1, dtype=torch.float64), "at least"),
+                      (torch.zeros((15, 16), dtype=torch.float64)[:, :8], "contiguous")):
+        with pytest.raises(ValueError, match=what):
+            fa._dev(bad, torch.float64, 15 * 8, "A_out")
+    with pytest.raises(ValueError, match="CUDA"):
+        fa._dev(ok, torch.float64, 15 * 8, "A_out")
+    with pytest.raises(TypeError):
+        fa._dev([0.0] * 120, torch.float64, 120, "A_out")
+    # the sizes the IRLS entry points ask of their optional outputs: p*m, p, workers, iters, 1
+    c = torch.zeros(15, dtype=torch.float32)
+    cases = dict(A_out=torch.zeros(15 * 8 - 1, dtype=torch.float64), w_out=torch.zeros(14, dtype=torch.float64),
+                 obj_out=torch.zeros(9, dtype=torch.float64), status=torch.zeros(1, dtype=torch.int64))
+    for name, bad in cases.items():
+        kw = dict(A_out=None, c_out=c, w_out=None, obj_out=None, status=None)
+        kw[name] = bad
+        with pytest.raises(ValueError, match=name):
+            fa._irls_outputs(None, 15, 8, 10, 15, **kw)
+    K = torch.zeros((15, 15), dtype=torch.float64)
+    for call in (lambda: fa.fa_irls(K, 8, 0.0, 10), lambda: fa.fa_irls(K[:, :14], 8, 0.0, 10),
+                 lambda: fa.fa_gram(torch.zeros((4, 10))), lambda: fa.fa_combine(torch.zeros((4, 10)), c)):
+        with pytest.raises(ValueError):
+            call()
+
+
 def test_package_refuses_to_import_without_its_library(tmp_path):
     """There is no CPU fallback: without libfa_b200.so the import itself fails."""
     pkg = tmp_path / "paper_2302_05865_b200"

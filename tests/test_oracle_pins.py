@@ -584,3 +584,65 @@ def test_beta_arguments():
     for bad in (dict(alpha=0.0), dict(alpha=1.5), dict(beta=0.0), dict(beta=1.2)):
         with pytest.raises(ValueError):
             fo.fa_aggregate(G, 2, **bad)
+
+
+# ---- comparison helper: the relative L2 error every aggregate-parity assertion is stated in ----------
+
+def test_relative_l2_error_on_hand_computed_cases():
+    assert fo.rel_l2([3.0, 4.0], [0.0, 0.0]) == 5.0                       # zero reference: the plain norm
+    assert abs(fo.rel_l2([1.0, 0.0], [0.0, 1.0]) - np.sqrt(2.0)) < 1e-15   # ||(1,-1)|| / ||(0,1)||
+    assert abs(fo.rel_l2([1.0, 2.0], [1.0, 1.0]) - 1.0 / np.sqrt(2.0)) < 1e-15
+    a, b = np.array([2.0, -1.0, 0.5]), np.array([1.0, 1.0, 1.0])
+    # the denominator is the SECOND argument: scaling it by 10 (and the difference with it) ...
+    assert abs(fo.rel_l2(10 * a, 10 * b) - fo.rel_l2(a, b)) < 1e-15
+    # ... and the measure is not symmetric
+    assert abs(fo.rel_l2(a, b) - np.sqrt(1.0 + 4.0 + 0.25) / np.sqrt(3.0)) < 1e-15
+    assert abs(fo.rel_l2(b, a) - np.sqrt(1.0 + 4.0 + 0.25) / np.sqrt(4.0 + 1.0 + 0.25)) < 1e-15
+    assert fo.rel_l2(b, b) == 0.0
+
+
+# ---- the any-n (column-blocked) form of the iteration -------------------------------------------------
+
+@pytest.mark.parametrize("p,n,m,lam,iters,block", [(9, 1000, 4, 0.2, 7, 128), (15, 700, 8, 0.01, 10, 97),
+                                                  (6, 50, 3, 0.0, 5, 7), (7, 333, 3, 0.3, 6, 1 << 16)])
+def test_blocked_iteration_equals_the_plain_one(p, n, m, lam, iters, block):
+    G = noisy_mean(p, n, 70 + p, sigma=0.5, outliers=2, scale_spread=True)
+    if p >= 7:
+        G[1] = G[0]                # an identical pair
+        G[p - 1] = 0.0             # a zero gradient
+    plain = fo.fa_aggregate(G, m, lam, iters)
+    for threads in (1, 3):
+        blk = fo.fa_aggregate_blocked(G, m, lam, iters, block=block, threads=threads)
+        assert blk["k"] == plain["Y"].shape[1]
+        assert np.allclose(blk["objective"], plain["objective"], rtol=0, atol=1e-10)
+        assert np.allclose(blk["u"], plain["u"], rtol=0, atol=1e-10)
+        assert np.allclose(blk["w"], plain["w"], rtol=1e-8, atol=0)
+        assert fo.rel_l2(blk["d"], plain["d"]) < 1e-10
+        assert blk["yty_err"] < 1e-10
+        # Z = G Y of the blocked run against the plain run's Y: cosines of the principal angles
+        # are the singular values of Y_plain^T Y_blocked, and Y_blocked^T g_i = Z[i]
+        Yb_coords = np.linalg.lstsq(G.T, plain["Y"], rcond=None)[0]      # Y_plain = G^T A (Y lies in span G)
+        cross = Yb_coords.T @ blk["Z"]                                    # = Y_plain^T Y_blocked
+        assert np.allclose(np.linalg.svd(cross, compute_uv=False), 1.0, atol=1e-9)
+        assert np.allclose(blk["K"], G @ G.T, rtol=1e-12)
+
+
+def test_blocked_iteration_returns_sampled_aggregate_and_its_norm():
+    G = noisy_mean(8, 500, 81, sigma=0.5, outliers=1)
+    full = fo.fa_aggregate_blocked(G, 3, 0.1, 4, block=64)
+    idx = np.array([0, 499, 63, 64, 65, 250, 250])
+    part = fo.fa_aggregate_blocked(G, 3, 0.1, 4, block=64, sample=idx)
+    assert np.array_equal(part["d_sample"], full["d"][idx])
+    assert abs(part["d_norm"] - np.linalg.norm(full["d"])) < 1e-12 * np.linalg.norm(full["d"])
+    assert "d" not in part
+
+
+def test_blocked_iteration_widens_the_stored_type_block_by_block():
+    G32 = noisy_mean(6, 300, 82, sigma=0.5, outliers=1).astype(np.float32)
+    calls = []
+    def widen(x):
+        calls.append(x.shape[1])
+        return x.astype(np.float64)
+    a = fo.fa_aggregate_blocked(G32, 3, 0.1, 3, block=100, widen=widen)
+    b = fo.fa_aggregate(G32.astype(np.float64), 3, 0.1, 3)
+    assert max(calls) == 100 and fo.rel_l2(a["d"], b["d"]) < 1e-10
