@@ -6,7 +6,7 @@
 
 namespace fa {
 
-template <int NT>
+template <int NT, int LD>
 __global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   extern __shared__ __align__(16) unsigned char irls_smem[];
   fa_irls::Ctx ctx{(int)threadIdx.x, (int)blockDim.x};
@@ -14,32 +14,35 @@ __global__ void __launch_bounds__(NT, 1) irls_kernel(IrlsArgs a) {
   fa_irls::Smem s;
   fa_irls::carve(s, irls_smem, a.p, ctx.nt);
   fa_irls::Outputs o{a.A, a.c, a.w, a.obj, a.S, a.status, a.rounds};
-  const int st = fa_irls::run<(NT > 192)>(ctx, s, K, a.p, a.m, a.lambda, a.a, a.iters, a.start_from_A, a.A0, a.tol, o,
+  const int st = fa_irls::run<LD>(ctx, s, K, a.p, a.m, a.lambda, a.a, a.iters, a.start_from_A, a.A0, a.tol, o,
                                            a.workers, a.counts, a.cb, a.ca);
   if (st && a.status && ctx.tid == 0) atomicOr(a.status, st);
 }
 
-template <int NT>
+template <int NT, int LD>
 static cudaError_t launch_nt(const IrlsArgs& a, cudaStream_t st) {
   const size_t smem = fa_irls::smem_bytes(a.p, NT);
-  cudaError_t e = cudaFuncSetAttribute(irls_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(irls_kernel<NT, LD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  irls_kernel<NT><<<1, NT, smem, st>>>(a);
+  irls_kernel<NT, LD><<<1, NT, smem, st>>>(a);
   return cudaGetLastError();
 }
 
 // One thread per Jacobi work item where the block size allows it: (p/2)^2 2x2 blocks plus
 // p * p/2 eigenvector row pairs.
 cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
+#ifndef FA_IRLS_NT16
+#define FA_IRLS_NT16 256
+#endif
 #ifndef FA_IRLS_NT32
 #define FA_IRLS_NT32 512
 #endif
 #ifndef FA_IRLS_NT64
 #define FA_IRLS_NT64 512
 #endif
-  if (a.p <= 16) return launch_nt<192>(a, st);
-  if (a.p <= 32) return launch_nt<FA_IRLS_NT32>(a, st);
-  return launch_nt<FA_IRLS_NT64>(a, st);
+  if (a.p <= 16) return launch_nt<FA_IRLS_NT16, 20>(a, st);
+  if (a.p <= 32) return launch_nt<FA_IRLS_NT32, 36>(a, st);
+  return launch_nt<FA_IRLS_NT64, 68>(a, st);
 }
 
 }  // namespace fa

@@ -9,14 +9,15 @@
 //     (n x r) has orthonormal columns with Q^T g_i = f_i.
 // A subspace Y = Q Z is represented by Z (r x m); in gradient coordinates Y = G A with
 // A = D^-1 V L^(-1/2) Z.  Each round forms T = sum w_i f_i f_i^T + sum w_ij (f_i-f_j)(f_i-f_j)^T
-// = F M F^T, diagonalises it by Jacobi (started in the previous round's eigenbasis, where T is
-// already nearly diagonal), keeps the m leading eigenvectors and evaluates the terms under the
-// square roots of Eq. (5) as squared residual norms, i.e. as sums of squares over the discarded
-// eigen-directions -- no "1 - x" cancellation.
+// = F M F^T in the previous round's eigenbasis and diagonalises it: cyclic Jacobi sweeps while T is
+// far from diagonal, then a matrix-product refinement of the eigenvectors that squares the error
+// per step at about a tenth of the cost of a sweep (refine_eig below).  The m leading eigenvectors
+// are kept and the terms under the square roots of Eq. (5) are evaluated as squared residual norms,
+// i.e. as sums of squares over the discarded eigen-directions -- no "1 - x" cancellation.
 //
 // The code is written as phases separated by block barriers, every phase a strided loop over
-// independent items, so that it can also be compiled for the host with one "thread" (used to
-// debug the arithmetic without a GPU).
+// independent items, so that it also compiles for the host with one "thread" (FA_IRLS_HOST): the
+// CPU test suite runs that build against the CPU reference implementation.
 #pragma once
 
 #include <math.h>
@@ -62,6 +63,9 @@ constexpr double kRankRel = 1e-12;     // eigenvalue <= this * largest: directio
 constexpr double kJacobiTol = 1e-17;   // rotate when |a_pq| > tol * sqrt(|a_pp a_qq|)
 constexpr double kJacobiBig = 1e-6;    // sweep again while some rotated |a_pq| exceeded this (relative)
 constexpr int kMaxSweeps = 40;
+constexpr double kRefineTheta = 0.3;   // refinement is tried when every |T_ij| <= this * |T_jj - T_ii|
+constexpr double kRefineStop = 1e-8;   // ... and has converged when a step's largest correction is below this
+constexpr int kMaxRefine = 8;          // steps after which a refinement that has not converged is given up
 constexpr int kMaxP = 64;
 
 constexpr int ST_NONFINITE = 1, ST_RANK0 = 2, ST_RANK_LT_M = 4, ST_EIG_SWEEPS = 8;
@@ -75,12 +79,40 @@ struct Ctx {
 #endif
 };
 
-// Shared-memory image.  Matrices are (pp x ld) doubles, pp = p rounded up to even, ld odd.
+// x / d for 0 <= x < 65536 and 1 <= d <= 64 without an integer division (a division by a run-time
+// value has a latency of about 75 cycles on this GPU, which is a fifth of a whole phase here): with
+// mul = ceil(2^32 / d) the high word of x * mul is the quotient exactly for these ranges.
+struct FastDiv { unsigned mul; int d; };
+FA_HD FastDiv make_div(int d) {
+  FastDiv f;
+  f.d = d < 1 ? 1 : d;
+  f.mul = f.d == 1 ? 0u : (unsigned)((0x100000000ULL + (unsigned long long)f.d - 1ULL) / (unsigned long long)f.d);
+  return f;
+}
+FA_FN int fast_div(int x, const FastDiv& f) {
+#ifndef FA_IRLS_HOST
+  return f.d == 1 ? x : (int)__umulhi((unsigned)x, f.mul);
+#else
+  return x / f.d;
+#endif
+}
+
+// Leading dimension of every matrix buffer: a compile-time constant per kernel instantiation (20, 36
+// or 68 doubles for up to 16, 32, 64 rows), which turns the element offsets of the unrolled inner
+// loops into immediates.  It is 4 modulo 16: the sixteen lanes of a half-warp that load a tensor-core
+// fragment (4 rows x 4 consecutive elements, or the transpose) then hit sixteen different bank pairs.
+constexpr int kLdPad = 4;
+FA_HD int leading_dim(int p) { return (p <= 16 ? 16 : (p <= 32 ? 32 : 64)) + kLdPad; }
+
+// Shared-memory image.  Matrices are (ld - kLdPad) x ld doubles.
 struct Smem {
   double *T, *J, *P, *M, *Aacc, *tmp;   // six matrix buffers, rotated by pointer swaps
   double *kd, *dinv, *fn, *u, *w, *wused, *ev, *red;
+  double *lam, *rdiag;                   // refinement: eigenvalue estimates, diagonal of I - X^T X
   double *rc, *rs;                       // rotation cos / sin per pair
   int *ra, *rb, *ord;                    // rotation indices per pair, sort order
+  int *piv;                              // pivot column of every step of the factorisation
+  unsigned short* pairs;                 // (i << 8) | j of the q-th worker pair i < j (see tri_pair)
   int *flags;                            // [0],[3] rotated-this-sweep (by sweep parity), [1] scratch
   // several gradients per worker (nw > 0): per-worker trace, value, weight, weight in use, 1/k_i;
   // grp[row] = worker of a row, first[i] = first row of worker i
@@ -88,19 +120,22 @@ struct Smem {
   int *grp, *first;
   int nw;
   int ld;
+  int count_sweeps, count_refinements;   // work done by the eigensolver in this call (diagnostics)
+  FastDiv div_r, div_p, div_tr, div_tp;  // by the rank r, by p, by their numbers of 8-wide tiles
+  int max_calls, sum_calls;              // block_max / block_sum calls so far (parity picks the exchange slots)
 };
 
 FA_HD size_t smem_bytes(int p, int nt) {
-  int pp = (p + 1) & ~1;
-  int ld = pp + 1;
-  size_t doubles = (size_t)6 * pp * ld + (size_t)12 * pp + nt + 2 * (pp / 2 + 1);
-  size_t ints = (size_t)2 * (pp / 2 + 1) + 3 * pp + 8;
+  int ld = leading_dim(p);
+  int pp = ld - kLdPad;
+  size_t doubles = (size_t)6 * pp * ld + (size_t)14 * pp + (nt < 128 ? 128 : nt) + 2 * (pp / 2 + 1);
+  size_t ints = (size_t)2 * (pp / 2 + 1) + 4 * pp + 8 + (size_t)(pp * (pp - 1) / 2 + 1) / 2;
   return doubles * sizeof(double) + ints * sizeof(int) + 64;
 }
 
 FA_FN void carve(Smem& s, void* base, int p, int nt) {
-  int pp = (p + 1) & ~1;
-  int ld = pp + 1;
+  int ld = leading_dim(p);
+  int pp = ld - kLdPad;
   double* d = reinterpret_cast<double*>(base);
   s.ld = ld;
   s.T = d; d += (size_t)pp * ld;
@@ -112,30 +147,230 @@ FA_FN void carve(Smem& s, void* base, int p, int nt) {
   s.kd = d; d += pp; s.dinv = d; d += pp; s.fn = d; d += pp; s.u = d; d += pp;
   s.w = d; d += pp; s.wused = d; d += pp; s.ev = d; d += pp;
   s.gtr = d; d += pp; s.gu = d; d += pp; s.gw = d; d += pp; s.gwused = d; d += pp; s.ginv = d; d += pp;
-  s.red = d; d += nt;
+  s.lam = d; d += pp; s.rdiag = d; d += pp;
+  s.red = d; d += (nt < 128 ? 128 : nt);
   s.rc = d; d += pp / 2 + 1; s.rs = d; d += pp / 2 + 1;
   int* q = reinterpret_cast<int*>(d);
   s.ra = q; q += pp / 2 + 1; s.rb = q; q += pp / 2 + 1; s.ord = q; q += pp; s.grp = q; q += pp;
-  s.first = q; q += pp; s.flags = q;
+  s.first = q; q += pp; s.piv = q; q += pp; s.flags = q; q += 8;
+  s.pairs = reinterpret_cast<unsigned short*>(q);
   s.nw = 0;
+  s.count_sweeps = 0; s.count_refinements = 0;
+  s.div_r = s.div_p = s.div_tr = s.div_tp = make_div(1);
+  s.max_calls = 0; s.sum_calls = 0;
 }
 
-// Deterministic block-wide sum; every thread gets the result.
-FA_FN double block_sum(const Ctx& c, const Smem& s, double v) {
+// Deterministic block-wide sum; every thread gets the result.  One barrier: the exchange slots
+// alternate between calls (see block_max), and every thread adds the warps' sums in the same order.
+FA_FN double block_sum(const Ctx& c, Smem& s, double v) {
 #ifndef FA_IRLS_HOST
   for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
-  c.sync();                                // s.red may still be read from a previous call
-  if ((c.tid & 31) == 0) s.red[c.tid >> 5] = v;
+  double* slots = s.red + 64 + ((s.sum_calls++ & 1) ? 32 : 0);
+  if ((c.tid & 31) == 0) slots[c.tid >> 5] = v;
   c.sync();
   double tot = 0.0;
-  int nw = (c.nt + 31) >> 5;
-  for (int k = 0; k < nw; ++k) tot += s.red[k];
+  const int nw = c.nt >> 5;
+  for (int k = 0; k < nw; ++k) tot += slots[k];
   return tot;
 #else
   (void)c; (void)s;
   return v;
 #endif
 }
+
+// Block-wide maximum of non-negative finite values; every thread gets the result, truncated to the
+// upper 32 bits of the double (about six digits) -- it only feeds threshold decisions, and every
+// thread takes the same ones.  Non-negative doubles order like their upper words, so the reduction
+// runs on integers: one warp reduction, one shared-memory exchange, one barrier (the exchange slots
+// alternate between calls, which keeps a slow warp's reads apart from the next call's writes).
+FA_FN double block_max(const Ctx& c, Smem& s, double v) {
+#ifndef FA_IRLS_HOST
+  const unsigned hi = __reduce_max_sync(0xffffffffu, (unsigned)__double2hiint(v));
+  unsigned* slots = reinterpret_cast<unsigned*>(s.red) + ((s.max_calls++ & 1) ? 32 : 0);
+  if ((c.tid & 31) == 0) slots[c.tid >> 5] = hi;
+  c.sync();
+  unsigned m = 0u;
+  const int nw = c.nt >> 5;
+  for (int k = 0; k < nw; ++k) m = max(m, slots[k]);
+  return __hiloint2double((int)m, 0);
+#else
+  (void)c; (void)s;
+  return v;
+#endif
+}
+
+// sum_k a[k * SA] * b[k * SB] over k < n <= NMAX.  The phases of this kernel are latency-bound (few
+// warps on one SM: a shared-memory load takes about 29 cycles, a dependent fp64 FMA 8), so the
+// operands of eight terms are loaded before the first product and two running sums are kept.  The
+// strides are compile-time constants (1 or the leading dimension): the loads of a chunk are one
+// base register plus immediates.  Up to 16 terms the chunks are unrolled and the loads predicated.
+template <int SA, int SB, int NMAX>
+FA_FN double dot(const double* a, const double* b, int n) {
+  constexpr int CH = 8;
+  double acc0 = 0.0, acc1 = 0.0;
+  if (NMAX <= 16) {
+#pragma unroll
+    for (int k0 = 0; k0 < NMAX; k0 += CH) {
+      double x[CH], y[CH];
+#pragma unroll
+      for (int u = 0; u < CH; ++u) {
+        const bool ok = k0 + u < n;
+        x[u] = ok ? a[(k0 + u) * SA] : 0.0; y[u] = ok ? b[(k0 + u) * SB] : 0.0;
+      }
+#pragma unroll
+      for (int u = 0; u < CH; u += 2) { acc0 = fma(x[u], y[u], acc0); acc1 = fma(x[u + 1], y[u + 1], acc1); }
+    }
+  } else {
+    for (int k0 = 0; k0 < n; k0 += CH, a += CH * SA, b += CH * SB) {
+      double x[CH], y[CH];
+#pragma unroll
+      for (int u = 0; u < CH; ++u) {
+        const bool ok = k0 + u < n;
+        x[u] = ok ? a[u * SA] : 0.0; y[u] = ok ? b[u * SB] : 0.0;
+      }
+#pragma unroll
+      for (int u = 0; u < CH; u += 2) { acc0 = fma(x[u], y[u], acc0); acc1 = fma(x[u + 1], y[u + 1], acc1); }
+    }
+  }
+  return acc0 + acc1;
+}
+
+// sum_k w[k] * a[k * SA] * b[k * SB] over k < n (same scheme).
+template <int SA, int SB, int NMAX>
+FA_FN double dot_weighted(const double* w, const double* a, const double* b, int n) {
+  constexpr int CH = 8;
+  double acc0 = 0.0, acc1 = 0.0;
+  for (int k0 = 0; k0 < n; k0 += CH, w += CH, a += CH * SA, b += CH * SB) {
+    double x[CH], y[CH];
+#pragma unroll
+    for (int u = 0; u < CH; ++u) {
+      const bool ok = k0 + u < n;
+      x[u] = ok ? w[u] * a[u * SA] : 0.0; y[u] = ok ? b[u * SB] : 0.0;
+    }
+#pragma unroll
+    for (int u = 0; u < CH; u += 2) { acc0 = fma(x[u], y[u], acc0); acc1 = fma(x[u + 1], y[u + 1], acc1); }
+  }
+  return acc0 + acc1;
+}
+
+// sum_k (a[k * ST] - b[k * ST])^2 over k in [0, n) and over k in [k0, n): squared distance of two
+// columns of a coordinate matrix, and of their parts in the discarded directions.
+template <int ST>
+FA_FN void diff_sq(const double* a, const double* b, int k0, int n, double& all, double& tail) {
+  constexpr int CH = 8;
+  double s0 = 0.0, s1 = 0.0, t0 = 0.0, t1 = 0.0;
+  for (int kb = 0; kb < n; kb += CH, a += CH * ST, b += CH * ST) {
+    double v[CH];
+#pragma unroll
+    for (int u = 0; u < CH; ++u) v[u] = (kb + u < n) ? a[u * ST] - b[u * ST] : 0.0;
+#pragma unroll
+    for (int u = 0; u < CH; u += 2) {
+      const double q0 = v[u] * v[u], q1 = v[u + 1] * v[u + 1];
+      s0 += q0; s1 += q1;
+      t0 += (kb + u >= k0) ? q0 : 0.0; t1 += (kb + u + 1 >= k0) ? q1 : 0.0;
+    }
+  }
+  all = s0 + s1; tail = t0 + t1;
+}
+
+// C = A B for small fp64 matrices (M x K times K x N) held in shared memory, on the fp64 tensor-core
+// instruction mma.m8n8k4: one warp per 8 x 8 tile of C, 256 multiply-adds per instruction with one
+// element of A and one of B per lane.  With one output element per thread every multiply-add needs
+// two shared-memory loads, and a 64-bit load instruction occupies the shared-memory pipe for two
+// cycles whatever its addresses: a 49 x 49 x 49 product took 16,500 cycles that way and takes about
+// a third of it this way (14 x 14 x 14: 690 -> below 400).
+//   A_ik = A[imap(i) * SAI + k * SAK],  B_kj = B[k * SBK + jmap(j) * SBJ]  (strides are 1 or the leading
+//   dimension, compile-time; imap / jmap are optional index lists, e.g. a sort order, null = identity)
+//   epi(i, j, v)  : consumes C_ij; called once per element in range
+//   dtn           : FastDiv by the number of column tiles, (N + 7) / 8
+//   first_warp    : the tiles go to warps first_warp, first_warp + 1, ... (mod the warp count), so
+//                   that two products of one phase use different warps
+// Fragments are loaded without bounds checks and masked afterwards: every index they can reach
+// (below the next multiple of 8 of M and N, of 16 of K) lies inside the (ld - kLdPad) x ld buffers.
+// All threads of the block must call it (whole warps execute the instruction); the number of warps
+// is a power of two.  The host build runs the plain triple loop.
+#ifndef FA_IRLS_HOST
+__device__ __forceinline__ void fa_dmma(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+}
+#endif
+
+template <int SAI, int SAK, int SBK, int SBJ, class EP>
+FA_FN void matmul(const Ctx& c, int M, int N, int K, const FastDiv& dtn, const double* A, const double* B, EP epi,
+                  int first_warp = 0, const int* imap = nullptr, const int* jmap = nullptr) {
+#ifndef FA_IRLS_HOST
+  const int lane = c.tid & 31, nwarp = c.nt >> 5;
+  const int warp = ((c.tid >> 5) - first_warp) & (nwarp - 1);
+  const int tn = (N + 7) >> 3, tiles = ((M + 7) >> 3) * tn;
+  const int fr = lane >> 2, fk = lane & 3;          // fragment coordinates: A (row fr, k fk), B (k fk, column fr)
+  for (int t = warp; t < tiles; t += nwarp) {
+    const int ti = fast_div(t, dtn);
+    const int i0 = ti * 8, j0 = (t - ti * tn) * 8;
+    const int i = i0 + fr, j = j0 + fr;
+    const bool iok = i < M, jok = j < N;
+    const int ia = imap ? imap[iok ? i : 0] : i, jb = jmap ? jmap[jok ? j : 0] : j;
+    const double* ap = A + ia * SAI + fk * SAK;
+    const double* bp = B + fk * SBK + jb * SBJ;
+    double d0 = 0.0, d1 = 0.0, e0 = 0.0, e1 = 0.0;  // two chains of dependent instructions, added at the end
+    for (int k0 = 0; k0 < K; k0 += 16, ap += 16 * SAK, bp += 16 * SBK) {
+      double a[4], b[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { a[u] = ap[4 * u * SAK]; b[u] = bp[4 * u * SBK]; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool kok = k0 + 4 * u + fk < K;
+        a[u] = (iok && kok) ? a[u] : 0.0;
+        b[u] = (jok && kok) ? b[u] : 0.0;
+      }
+      fa_dmma(d0, d1, a[0], b[0]);
+      fa_dmma(e0, e1, a[1], b[1]);
+      if (k0 + 8 < K) {                              // uniform in the warp
+        fa_dmma(d0, d1, a[2], b[2]);
+        fa_dmma(e0, e1, a[3], b[3]);
+      }
+    }
+    const int jc = j0 + 2 * fk;
+    if (iok) {
+      if (jc < N) epi(i, jc, d0 + e0);
+      if (jc + 1 < N) epi(i, jc + 1, d1 + e1);
+    }
+  }
+#else
+  (void)first_warp; (void)dtn;
+  for (int idx = c.tid; idx < M * N; idx += c.nt) {
+    const int i = idx / N, j = idx - i * N;
+    const int ia = imap ? imap[i] : i, jb = jmap ? jmap[j] : j;
+    double acc = 0.0;
+    for (int k = 0; k < K; ++k) acc += A[ia * SAI + k * SAK] * B[k * SBK + jb * SBJ];
+    epi(i, j, acc);
+  }
+#endif
+}
+
+// The q-th pair (i, j), i <= j, in the order (0,0) (0,1) (1,1) (0,2) (1,2) (2,2) ...: q = j (j + 1) / 2 + i.
+// The numbering does not depend on the matrix size.
+FA_FN void tri_pair(int q, int& i, int& j) {
+  int jj = (int)((sqrtf(8.0f * (float)q + 1.0f) - 1.0f) * 0.5f);   // within one of the answer; fixed up below
+  while (jj * (jj + 1) / 2 > q) --jj;
+  while ((jj + 1) * (jj + 2) / 2 <= q) ++jj;
+  j = jj; i = q - jj * (jj + 1) / 2;
+}
+
+#ifndef FA_IRLS_HOST
+// 1 / x for normal x: hardware approximation and two Newton steps (relative error ~1e-15 at best;
+// it scales corrections that are themselves iterated on).
+__device__ __forceinline__ double fa_fast_rcp(double x) {
+  double y;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+  y = fma(y, fma(-x, y, 1.0), y);
+  y = fma(y, fma(-x, y, 1.0), y);
+  return y;
+}
+#define FA_RCP(x) fa_fast_rcp(x)
+#else
+#define FA_RCP(x) (1.0 / (x))
+#endif
 
 // Rotation (cs, sn) for a pair with diagonal entries app, aqq and off-diagonal entry apq; identity
 // for entries at rounding level.  From the double angle, without division:
@@ -189,11 +424,12 @@ FA_FN int systolic_next(int x, int np) {
 }
 
 // Cyclic Jacobi, all pairs of a round in parallel.  T (dim x dim, symmetric, both halves stored, rows
-// and columns dim..pp-1 zero) is driven to diagonal form; J accumulates the rotations (J <- J * R).
-// A pair is rotated whenever its off-diagonal entry is above rounding level; sweeping stops after
-// the first sweep in which no rotated entry exceeded kJacobiBig relative to its diagonal: that
-// sweep's rotations leave entries of the order of its square (quadratic convergence of the cyclic
-// method), i.e. below rounding level.
+// and columns dim..pp-1 zero) is driven towards diagonal form; J accumulates the rotations (J <- J * R).
+// A pair is rotated whenever its off-diagonal entry is above rounding level.  At most `max_sweeps`
+// sweeps are made; sweeping also stops after the first sweep in which no rotated entry exceeded
+// kJacobiBig relative to its diagonal: that sweep's rotations leave entries of the order of its
+// square (quadratic convergence of the cyclic method), i.e. below rounding level.  *big_out tells
+// whether the last sweep made still saw such an entry (T is then not yet diagonal).
 //
 // The data MOVES instead of the pairing (Brent-Luk systolic arrangement): a round rotates the pairs
 // at the fixed positions (k, np + k) and stores rows and columns (and the columns of J) at their
@@ -201,16 +437,18 @@ FA_FN int systolic_next(int x, int np) {
 // 2x2 blocks of T and (row, pair) items of J for the whole solve, all its offsets are worked out
 // once before the first sweep, and all its loads go out together at the top of a round -- what a
 // round costs here is the number of dependent instructions a warp has to issue.
-//   * up to 8 pairs (dim <= 16): one item per thread; each thread works out the one or two
-//     rotations it needs itself: one barrier per round and nothing else between threads;
-//   * more pairs: several items per thread; the rotations are worked out once by the first np
-//     threads and published in shared memory (a second barrier per round).
+//   * up to 8 pairs (dim <= 16): one item per thread; each lane works out the rotation of its
+//     column pair itself and gets the one of its row pair from another lane of its warp by a
+//     shuffle: one barrier per round and nothing else between threads;
+//   * more pairs (jacobi_large): several items per thread; every warp works out all rotations
+//     (lane q: pair q) and the items fetch theirs by shuffles -- still one barrier per round.
 // A full sweep (pp - 1 rounds) returns every index to its own position, and sweeps are never cut
 // short.  On return *Tio / *Jio point at the buffers that hold the results.  Returns the sweeps made.
 // Up to 8 pairs on the device; any size on the host.
+template <int LD>
 FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
-                       int dim, int jrows) {
-  const int ld = s.ld;
+                       int dim, int jrows, int max_sweeps, int* big_out) {
+  constexpr int ld = LD;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
   double* T = *Tio;
@@ -233,12 +471,11 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       it.x0 = a * ld + cc; it.x1 = a * ld + d; it.x2 = b * ld + cc; it.x3 = b * ld + d;
       it.z0 = pa * ld + pc; it.z1 = pa * ld + pd; it.z2 = pb * ld + pc; it.z3 = pb * ld + pd;
 #ifndef FA_IRLS_HOST
-      // a lane of this warp whose own (column) pair is k hands over the row rotation
+      // a lane of this warp whose own (column) pair is k hands over the row rotation: the item with
+      // number o has column pair o mod np (nb2 is a multiple of np), so the first such lane is
       const int w0 = idx & ~31;
-      for (int j = 0; j < 32; ++j) {
-        const int o = w0 + j;
-        if (o < total2 && (o < nb2 ? o % np : (o - nb2) % np) == k) { it.ksrc = j; break; }
-      }
+      const int j = (k - w0 % np + np) % np;
+      if (j < 32 && w0 + j < total2) it.ksrc = j;
 #endif
     } else if (idx < total2) {
       const int q = idx - nb2;
@@ -251,11 +488,11 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       it.kaa = it.kbb = it.kab = it.x2 = it.x3 = it.z2 = it.z3 = 0;
     }
   }
-  int sweep = 0;
+  int sweep = 0, again = 0;
   // "large rotation in this sweep" flag, double-buffered by sweep parity (slots 0 and 3)
   if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
   c.sync();
-  for (; sweep < kMaxSweeps; ++sweep) {
+  for (; sweep < max_sweeps; ++sweep) {
     int* big = &s.flags[(sweep & 1) ? 3 : 0];
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
@@ -342,11 +579,12 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       { double* t = T; T = Tn; Tn = t; }
       { double* t = J; J = Jn; Jn = t; }
     }
-    const int again = *big;
+    again = *big;
     c.sync();
     if (!again) { ++sweep; break; }
   }
   *Tio = T; *Taltio = Tn; *Jio = J; *Jaltio = Jn;
+  *big_out = again;
   return sweep;
 }
 
@@ -355,10 +593,10 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
 // them) and (row, pair) items of J (kMJ).  Per item: the offset of its first element, the offsets
 // its results are stored at, and the pairs whose rotations it needs; offsets are below 2^16
 // (matrices of at most 64 x 65 doubles) and are kept two to a register.
-template <int kMT, int kMJ>
+template <int LD, int kMT, int kMJ>
 FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
-                       int dim, int jrows) {
-  const int ld = s.ld;
+                       int dim, int jrows, int max_sweeps, int* big_out) {
+  constexpr int ld = LD;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
   double* T = *Tio;
@@ -386,10 +624,10 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
     jdesc0[u] = (unsigned)(x * ld + l) | ((unsigned)l << 16);
     jdesc1[u] = (unsigned)(x * ld + systolic_next(l, np)) | ((unsigned)(x * ld + systolic_next(np + l, np)) << 16);
   }
-  int sweep = 0;
+  int sweep = 0, again = 0;
   if (c.tid == 0) { s.flags[0] = 0; s.flags[3] = 0; }
   c.sync();
-  for (; sweep < kMaxSweeps; ++sweep) {
+  for (; sweep < max_sweeps; ++sweep) {
     int* big = &s.flags[(sweep & 1) ? 3 : 0];
     if (c.tid == 0) s.flags[(sweep & 1) ? 0 : 3] = 0;
     for (int rd = 0; rd < pp - 1; ++rd) {
@@ -461,54 +699,160 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
       { double* t = T; T = Tn; Tn = t; }
       { double* t = J; J = Jn; Jn = t; }
     }
-    const int again = *big;
+    again = *big;
     c.sync();
     if (!again) { ++sweep; break; }
   }
   *Tio = T; *Taltio = Tn; *Jio = J; *Jaltio = Jn;
+  *big_out = again;
   return sweep;
 }
 #endif
 
-template <bool LARGE>
+template <int LD>
 FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio, int dim,
-                 int jrows) {
+                 int jrows, int max_sweeps, int* big_out) {
+  *big_out = 0;
   if (dim < 2) return 0;
 #ifndef FA_IRLS_HOST
   // item slots per thread are compile-time (slots without an item still cost their instructions):
   // one of each up to 16 pairs with 512 threads, two blocks and four J items up to 32 pairs
   const int np = (dim + 1) >> 1;
-  if (LARGE && np > 8) {
-    if (np * np <= c.nt && jrows * np <= c.nt) return jacobi_large<1, 1>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
-    return jacobi_large<2, 4>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
+  if (LD > 20 && np > 8) {
+    if (np * np <= c.nt && jrows * np <= c.nt)
+      return jacobi_large<LD, 1, 1>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+    return jacobi_large<LD, 2, 4>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
   }
 #endif
-  return jacobi_small(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows);
+  return jacobi_small<LD>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+}
+
+// Refinement of approximate eigenvectors by matrix products (the iterative refinement for the
+// symmetric eigenvalue decomposition of Ogita and Aishima, Japan J. Indust. Appl. Math. 35 (2018)):
+// for X (r x r, nearly orthogonal) with X^T T X nearly diagonal,
+//     Rm = I - X^T X,  S = X^T T X,  lam_i = S_ii / (1 - Rm_ii),
+//     E_ij = (S_ij + lam_j Rm_ij) / (lam_j - lam_i)  (i != j),  E_ii = Rm_ii / 2,   X <- X + X E
+// squares the distance of X from the exact orthogonal eigenvector matrix.  A step is four r x r
+// products (length-r dot products, independent of each other) against 2 (r - 1) dependent rotation
+// rounds for a Jacobi sweep.  It only converges from close by: |E_ij| must be well below one, which
+// near-equal eigenvalues with a sizeable coupling entry violate -- those stay with the Jacobi sweeps.
+//
+// Starts from X = I, i.e. in the basis T is given in; the first step then needs no products
+// (S = T, Rm = 0).  Returns 1 with X in s.J and the eigenvalue estimates on the diagonal of T when
+// the corrections went below kRefineStop; 0 (T untouched) when the first corrections are above
+// kRefineTheta, the steps stop contracting or kMaxRefine steps are not enough.  Uses s.J, s.tmp and
+// s.M as scratch (pointers may come back swapped).
+template <int LD>
+FA_FN int refine_eig(const Ctx& c, Smem& s, int r) {
+  constexpr int ld = LD;
+  const double* T = s.T;
+  double* X = s.J;       // current eigenvector estimate
+  double* E = s.tmp;     // T X, then the correction E
+  double* SR = s.M;      // S on and above the diagonal, Rm below it; becomes the next X
+  const int ntri = r * (r + 1) / 2;
+  // ---- first step from X = I
+  double part = 0.0;
+  for (int idx = c.tid; idx < r * r; idx += c.nt) {
+    const int i = fast_div(idx, s.div_r), j = idx - i * r;
+    double e = 0.0;
+    if (i != j) {
+      const double tij = T[i * ld + j], tii = T[i * ld + i], tjj = T[j * ld + j];
+      if (tij * tij > (kJacobiTol * kJacobiTol) * fabs(tii * tjj) && tij * tij > 1e-280) {
+        e = tij * FA_RCP(tjj - tii);                 // equal diagonal entries: Inf, refused below
+        part = fmax(part, fabs(e) <= 1.7e308 ? fabs(e) : 1.7e308);
+      }
+    }
+    X[i * ld + j] = (i == j) ? 1.0 : e;
+  }
+  double emax = block_max(c, s, part);               // its barrier also publishes X
+  if (!(emax <= kRefineTheta)) return 0;
+  for (int k = c.tid; k < r; k += c.nt) s.lam[k] = T[k * ld + k];
+  int steps = 1;
+  while (emax >= kRefineStop) {
+    if (steps > kMaxRefine) return 0;
+    const double prev = emax;
+    // ---- E <- T X
+    matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, T, X, [&](int i, int j, double v) { E[i * ld + j] = v; });
+    c.sync();
+    // ---- S = X^T (T X) on and above the diagonal, Rm = I - X^T X below it (its diagonal -> rdiag)
+    matmul<1, LD, LD, 1>(c, r, r, r, s.div_tr, X, E, [&](int i, int j, double v) { if (i <= j) SR[i * ld + j] = v; });
+    matmul<1, LD, LD, 1>(c, r, r, r, s.div_tr, X, X,
+                         [&](int i, int j, double v) { if (i == j) s.rdiag[i] = 1.0 - v; else if (i > j) SR[i * ld + j] = -v; },
+                         ((r + 7) >> 3) * ((r + 7) >> 3));
+    c.sync();
+    // ---- the correction.  lam_i = S_ii / (1 - Rm_ii) with the quotient expanded to second order:
+    // Rm_ii is of the order of the last correction squared.
+    part = 0.0;
+    for (int idx = c.tid; idx < r * r; idx += c.nt) {
+      const int i = fast_div(idx, s.div_r), j = idx - i * r;
+      const double rii = s.rdiag[i];
+      const double li = SR[i * ld + i] * fma(rii, 1.0 + rii, 1.0);
+      double e;
+      if (i == j) { e = 0.5 * rii; s.lam[i] = li; }
+      else {
+        const double rjj = s.rdiag[j];
+        const double lj = SR[j * ld + j] * fma(rjj, 1.0 + rjj, 1.0);
+        const double sij = (i < j) ? SR[i * ld + j] : SR[j * ld + i];
+        const double rij = (i < j) ? SR[j * ld + i] : SR[i * ld + j];
+        const double num = fma(lj, rij, sij);
+        if (num * num > (kJacobiTol * kJacobiTol) * fabs(li * lj) && num * num > 1e-280) {
+          e = num * FA_RCP(lj - li);
+          part = fmax(part, fabs(e) <= 1.7e308 ? fabs(e) : 1.7e308);
+        } else {
+          e = 0.5 * rij;                             // nothing to rotate: keep the pair orthogonal
+        }
+      }
+      E[i * ld + j] = e;
+    }
+    emax = block_max(c, s, part);                    // its barrier: every thread is done with SR, E is published
+    if (!(emax <= 0.5 * prev) && emax > 1e-12) return 0;
+    // ---- X <- X + X E  (into SR's buffer, which then changes roles with X's)
+    matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, X, E, [&](int i, int j, double v) { SR[i * ld + j] = X[i * ld + j] + v; });
+    c.sync();
+    { double* t = X; X = SR; SR = t; }
+    ++steps;
+  }
+  c.sync();
+  for (int k = c.tid; k < r; k += c.nt) s.T[k * ld + k] = s.lam[k];
+  s.J = X; s.M = SR;
+  s.count_refinements += steps;
+  c.sync();
+  return 1;
 }
 
 // ev[k] = T[k][k]; ord[q] = index of the q-th largest (ties by index).  All threads return
 // the number of eigenvalues > kRankRel * largest among the first `limit` in that order.
+// One phase: the thread of index k reads the whole diagonal, so it knows the rank of its own
+// entry and the largest one; the count is taken by the barrier that publishes ord and ev.
+template <int LD>
 FA_FN int sort_eigs(const Ctx& c, const Smem& s, const double* T, int dim, int limit) {
-  const int ld = s.ld;
-  for (int k = c.tid; k < dim; k += c.nt) s.ev[k] = T[k * ld + k];
-  c.sync();
+  constexpr int ld = LD;
+  const int lim = limit < dim ? limit : dim;
+  int mine = 0;
+#ifdef FA_IRLS_HOST
+  int keep = 0;
+#endif
   for (int k = c.tid; k < dim; k += c.nt) {
-    double e = s.ev[k];
+    const double e = T[k * ld + k];
+    double top = e;
     int rank = 0;
     for (int l = 0; l < dim; ++l) {
-      double o = s.ev[l];
+      const double o = T[l * ld + l];
       rank += (o > e || (o == e && l < k)) ? 1 : 0;
+      top = fmax(top, o);
     }
     s.ord[rank] = k;
+    s.ev[k] = e;
+    mine = (rank < lim && top > 0.0 && e > kRankRel * top) ? 1 : 0;
+#ifdef FA_IRLS_HOST
+    keep += mine;
+#endif
   }
-  c.sync();
-  double top = s.ev[s.ord[0]];
-  int keep = 0;
-  if (top > 0.0) {
-    int lim = limit < dim ? limit : dim;
-    for (int q = 0; q < lim; ++q) keep += (s.ev[s.ord[q]] > kRankRel * top) ? 1 : 0;
-  }
+#ifndef FA_IRLS_HOST
+  return __syncthreads_count(mine);
+#else
   return keep;
+#endif
 }
 
 // One term of the objective with value u (the quantity under the root in Eq. (5)): its
@@ -527,17 +871,17 @@ FA_FN void term_of(double u, double a, double& contrib, double& denom) {
 // cb, ca: the data term of worker i is cb (1 - v_i)^(1/a) + ca v_i^(1/a) -- a Beta(alpha, beta)
 // likelihood of the values with cb = 2 (1 - beta), ca = 2 (1 - alpha); Eq. (1) has alpha = 1,
 // beta = 1/2, i.e. cb = 1, ca = 0.  With ca > 0 a weight can be negative.
+template <int LD>
 FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
                                    double coef, bool uniform, double a, double cb = 1.0, double ca = 0.0) {
-  const int ld = s.ld;
+  constexpr int ld = LD;
   double part = 0.0;
   for (int i = c.tid; i < p; i += c.nt) {
     double ui = 0.0, wi = 0.0;
     if (s.dinv[i] != 0.0) {
       if (uniform) wi = 1.0;
       else {
-        double acc = 0.0;
-        for (int k = k0; k < r; ++k) { double v = Res[k * ld + i]; acc += v * v; }
+        const double acc = dot<LD, LD, LD - kLdPad>(Res + k0 * ld + i, Res + k0 * ld + i, r - k0);
         if (a == 2.0 && cb == 1.0 && ca == 0.0) {
           // the paper's square roots without a division or a square root: with y = 1/sqrt(acc fn),
           // sqrt(u) = acc y and 1/(fn sqrt(u)) = y
@@ -579,36 +923,37 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
   }
   c.sync();
   if (coef > 0.0) {
-    // off-diagonal entries M_ij = -2 w_ij (ordered pairs: each unordered pair counted twice)
-    for (int idx = c.tid; idx < p * p; idx += c.nt) {
-      int i = idx / p, j = idx - i * p;
-      if (i == j) continue;
-      double d2 = 0.0, res2 = 0.0;
-      for (int k = 0; k < r; ++k) { double v = s.P[k * ld + i] - s.P[k * ld + j]; d2 += v * v; }
+    // off-diagonal entries M_ij = M_ji = -2 w_ij (ordered pairs: each unordered pair counted twice, and
+    // twice in the objective); one item per unordered pair i < j
+    for (int idx = c.tid; idx < p * (p - 1) / 2; idx += c.nt) {
+      const int i = s.pairs[idx] >> 8, j = s.pairs[idx] & 255;
+      double d2, res2;
+      diff_sq<LD>(s.P + i, s.P + j, (Res == s.P) ? k0 : r, r, d2, res2);
       double wij = 0.0;
       if (d2 > kSamePairRel * (s.fn[i] + s.fn[j])) {
         if (uniform) wij = coef;
         else {
-          for (int k = k0; k < r; ++k) { double v = Res[k * ld + i] - Res[k * ld + j]; res2 += v * v; }
+          if (Res != s.P) { double all; diff_sq<LD>(Res + i, Res + j, k0, r, all, res2); }
           if (a == 2.0) {
             const double y = res2 > 0.0 ? FA_RSQRT(res2 * d2) : 0.0;     // sqrt(u) = res2 y, 1/(d2 sqrt(u)) = y
             const double contrib = res2 * y;
-            part += coef * contrib;
+            part += 2.0 * coef * contrib;
             wij = contrib >= kEps ? coef * y : coef / (d2 * kEps);
           } else {
             double contrib, denom;
             term_of(res2 / d2, a, contrib, denom);
-            part += coef * contrib;
+            part += 2.0 * coef * contrib;
             wij = coef / (d2 * denom);
           }
         }
       }
       s.M[i * ld + j] = -2.0 * wij;
+      s.M[j * ld + i] = -2.0 * wij;
     }
     c.sync();
     for (int i = c.tid; i < p; i += c.nt) {
       double acc = 0.0;
-      for (int j = 0; j < p; ++j) if (j != i) acc -= s.M[i * ld + j];
+      for (int j = 0; j < p; ++j) acc -= (j != i) ? s.M[i * ld + j] : 0.0;
       s.M[i * ld + i] = s.w[i] + acc;
     }
   }
@@ -621,9 +966,11 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
 // one weight per worker multiplies all of its rows, and the pair terms of the regulariser are taken
 // between the workers' mean gradients.  `p` is the number of rows.  s.T and s.J are scratch here
 // (mean coordinates of every worker: all of them, and the residual part).
+template <int LD>
 FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
                                            double coef, bool uniform, double a) {
-  const int ld = s.ld, nw = s.nw;
+  constexpr int ld = LD;
+  const int nw = s.nw;
   double* Fm = s.T;
   double* Rm = s.J;
   double part = 0.0;
@@ -724,21 +1071,22 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
 // first, and a rank-deficient one falls back to the uniform round.  tol >= 0: stop after round
 // t >= 2 once the objective moved by <= tol (remaining entries of o.obj repeat the last value).  nw > 0: the p rows belong to nw workers, cnt[i] consecutive rows each (o.w then has nw
 // entries); nw = 0: one gradient per worker.  Returns the status bits (same value in every thread).
-template <bool LARGE>
+template <int LD>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
               int start, const double* A0, double tol, const Outputs& o, int nw = 0,
               const unsigned char* cnt = nullptr, double cb = 1.0, double ca = 0.0) {
-  const int ld = s.ld;
+  constexpr int ld = LD;
   const int pp = (p + 1) & ~1;
   int status = 0;
 
   // ---- load K, reject non-finite input
   if (c.tid == 0) { s.flags[1] = 0; }
+  s.div_p = make_div(p);
   c.sync();
   for (int idx = c.tid; idx < pp * ld; idx += c.nt) { s.T[idx] = 0.0; s.J[idx] = 0.0; s.Aacc[idx] = 0.0; s.P[idx] = 0.0; s.M[idx] = 0.0; s.tmp[idx] = 0.0; }
   c.sync();
   for (int idx = c.tid; idx < p * p; idx += c.nt) {
-    int i = idx / p, j = idx - i * p;
+    const int i = fast_div(idx, s.div_p), j = idx - i * p;
     double v = K[idx];
     if (!(fabs(v) <= 1.7e308)) s.flags[1] = 1;
     s.T[i * ld + j] = v;
@@ -748,114 +1096,134 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     write_zero_outputs(c, o, p, m, iters, nw > 0 ? nw : p);
     return ST_NONFINITE;
   }
-  for (int i = c.tid; i < p; i += c.nt) s.kd[i] = s.T[i * ld + i];
-  c.sync();
   double kmax = 0.0;
-  for (int i = 0; i < p; ++i) kmax = fmax(kmax, s.kd[i]);
+  for (int i = 0; i < p; ++i) kmax = fmax(kmax, s.T[i * ld + i]);
   if (!(kmax > 0.0)) {
     write_zero_outputs(c, o, p, m, iters, nw > 0 ? nw : p);
     return ST_RANK0;
   }
-  for (int i = c.tid; i < p; i += c.nt)
-    s.dinv[i] = (s.kd[i] <= kZeroNormRel * kmax) ? 0.0 : 1.0 / sqrt(s.kd[i]);
+  for (int idx = c.tid; idx < p * (p - 1) / 2; idx += c.nt) {
+    int i, jm;
+    tri_pair(idx, i, jm);                         // i <= jm over p - 1 columns: the pair (i, jm + 1)
+    s.pairs[idx] = (unsigned short)((i << 8) | (jm + 1));
+  }
+  // kd = ||g_i||^2, dinv = 1 / ||g_i|| (0 for a zero gradient), fn (for now) = ||g_i||
+  for (int i = c.tid; i < p; i += c.nt) {
+    const double kii = s.T[i * ld + i];
+    const bool zero = kii <= kZeroNormRel * kmax;
+    const double nrm = zero ? 0.0 : sqrt(kii);
+    s.kd[i] = kii; s.fn[i] = nrm; s.dinv[i] = zero ? 0.0 : 1.0 / nrm;
+  }
   c.sync();
 
   // ---- Kt = D^-1 K D^-1 (symmetrised, unit diagonal) -> tmp
-  for (int idx = c.tid; idx < p * p; idx += c.nt) {
-    int i = idx / p, j = idx - i * p;
-    if (j < i) continue;
+  for (int idx = c.tid; idx < p * (p + 1) / 2; idx += c.nt) {
+    int i, j;
+    tri_pair(idx, i, j);
     double v = (i == j) ? (s.dinv[i] != 0.0 ? 1.0 : 0.0)
                         : 0.5 * (s.T[i * ld + j] + s.T[j * ld + i]) * s.dinv[i] * s.dinv[j];
     s.tmp[i * ld + j] = v; s.tmp[j * ld + i] = v;
   }
-  // remaining diagonal of the factorisation -> u; "already a pivot" marks -> ord (as flags)
+  // remaining diagonal of the factorisation -> u (and, on alternate steps, w: see below); ord[j] = 0
+  // while column j has not been a pivot, else 1 + the step at which it was
   for (int i = c.tid; i < p; i += c.nt) { s.u[i] = (s.dinv[i] != 0.0) ? 1.0 : 0.0; s.ord[i] = 0; }
   c.sync();
 
   // ---- Cholesky with complete pivoting, Kt = R^T R, R (r x p) kept in P with the original column
   // order: column i of R is the image f_i / ||g_i|| of worker i in R^r.  Stops when the largest
   // remaining diagonal entry is <= kRankRel (the diagonal of Kt is 1), which fixes the rank r.
+  // One barrier per step: the pivot is found by every warp for itself (a reduction on the upper
+  // words of the remaining diagonal -- values closer than six digits count as tied and the lowest
+  // index wins), and the thread of column j updates the column and its remaining diagonal entry.
+  // What a step writes must not be seen by a warp that is still searching in the same step: the
+  // remaining diagonal alternates between two arrays, and a pivot mark counts from the next step on.
   int r = 0;
   for (int k = 0; k < p; ++k) {
+    const double* ucur = (k & 1) ? s.w : s.u;
+    double* unext = (k & 1) ? s.u : s.w;
     int piv = -1;
-    double dmax = kRankRel;
 #ifndef FA_IRLS_HOST
-    if (p > 32) {
-      // every warp finds the pivot itself (two candidates per lane, butterfly); ties go to the lowest index
-      for (int j = (c.tid & 31); j < p; j += 32) {
-        const double dj = s.u[j];
-        if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
-      }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        const double od = __shfl_xor_sync(0xffffffffu, dmax, off);
-        const int oi = __shfl_xor_sync(0xffffffffu, piv, off);
-        if (od > dmax || (od == dmax && oi >= 0 && (piv < 0 || oi < piv))) { dmax = od; piv = oi; }
-      }
-    } else
-#endif
     {
-      for (int j = 0; j < p; ++j) {               // every thread scans; ties go to the lowest index
-        const double dj = s.u[j];
+      const int lane = c.tid & 31;
+      const int m0 = lane < p ? s.ord[lane] : 1, m1 = lane + 32 < p ? s.ord[lane + 32] : 1;
+      const double u0 = (m0 == 0 || m0 > k) ? ucur[lane < p ? lane : 0] : 0.0;
+      const double u1 = (m1 == 0 || m1 > k) ? ucur[lane + 32 < p ? lane + 32 : 0] : 0.0;
+      const unsigned h0 = (lane < p) ? (unsigned)__double2hiint(u0) : 0u;
+      const unsigned h1 = (lane + 32 < p) ? (unsigned)__double2hiint(u1) : 0u;
+      const unsigned best = __reduce_max_sync(0xffffffffu, max(h0, h1));
+      const unsigned cand = (h0 == best && lane < p) ? (unsigned)lane
+                                                     : ((h1 == best && lane + 32 < p) ? (unsigned)(lane + 32) : 64u);
+      const unsigned at = __reduce_min_sync(0xffffffffu, cand);
+      if (best > (unsigned)__double2hiint(kRankRel) && at < 64u) piv = (int)at;
+    }
+#else
+    {
+      double dmax = kRankRel;
+      for (int j = 0; j < p; ++j) {               // ties go to the lowest index
+        const double dj = ucur[j];
         if (s.ord[j] == 0 && dj > dmax) { dmax = dj; piv = j; }
       }
     }
+#endif
     if (piv < 0) break;
-    const double rinv = FA_RSQRT(dmax), rkk = dmax * rinv;   // dmax in (1e-12, 1]: a normal number
+    const double dpiv = ucur[piv];
+    if (!(dpiv > kRankRel)) break;                // (the upper-word test lets a value just below the cut through)
+    const double rinv = FA_RSQRT(dpiv), rkk = dpiv * rinv;   // dpiv in (1e-12, 1]: a normal number
     for (int j = c.tid; j < p; j += c.nt) {
-      double v;
-      if (j == piv) v = rkk;
-      else if (s.ord[j] != 0) v = 0.0;
+      const int mark = s.ord[j];
+      const bool done = mark != 0 && mark <= k;   // a pivot of an earlier step
+      double v, left = 0.0;
+      if (j == piv) { v = rkk; s.ord[j] = k + 1; s.piv[k] = piv; s.lam[k] = rinv; }
+      else if (done) v = 0.0;
       else {
-        double acc = s.tmp[piv * ld + j];
-        for (int l = 0; l < k; ++l) acc -= s.P[l * ld + piv] * s.P[l * ld + j];
-        v = acc * rinv;
+        v = (s.tmp[piv * ld + j] - dot<LD, LD, LD - kLdPad>(s.P + piv, s.P + j, k)) * rinv;
+        left = fmax(ucur[j] - v * v, 0.0);
       }
       s.P[k * ld + j] = v;
-    }
-    if (c.tid == 0) s.wused[k] = (double)piv;     // pivot order (exact small integers)
-    c.sync();
-    for (int j = c.tid; j < p; j += c.nt) {
-      if (j == piv) { s.ord[j] = 1; s.u[j] = 0.0; }
-      else if (s.ord[j] == 0) { const double v = s.P[k * ld + j]; s.u[j] = fmax(s.u[j] - v * v, 0.0); }
+      unext[j] = left;
     }
     c.sync();
     r = k + 1;
   }
+  s.div_r = make_div(r);
+  s.div_tr = make_div((r + 7) >> 3); s.div_tp = make_div((p + 7) >> 3);
 
   // ---- U = R11^-1 (R11 = pivot columns of R, upper triangular) by back substitution, one column
   // per thread -> J buffer.  Q = G D^-1 X with X[piv_a][:] = U[a][:] has orthonormal columns and
-  // Q^T g_i = f_i, so Aacc starts as D^-1 X (p x r).
+  // Q^T g_i = f_i, so Aacc starts as D^-1 X (p x r).  First the pivot columns are gathered (-> M),
+  // so that the sums below run over consecutive elements; 1 / R11_aa is the rinv of step a.
+  for (int idx = c.tid; idx < r * r; idx += c.nt) {
+    const int a = fast_div(idx, s.div_r), l = idx - a * r;
+    s.M[a * ld + l] = s.P[a * ld + s.piv[l]];
+  }
+  c.sync();
   for (int bcol = c.tid; bcol < r; bcol += c.nt) {
     for (int a = bcol; a >= 0; --a) {
-      const int pa = (int)s.wused[a];
-      double acc = (a == bcol) ? 1.0 : 0.0;
-      for (int l = a + 1; l <= bcol; ++l) acc -= s.P[a * ld + (int)s.wused[l]] * s.J[l * ld + bcol];
-      s.J[a * ld + bcol] = acc / s.P[a * ld + pa];
+      const double sum = dot<1, LD, LD - kLdPad>(s.M + a * ld + a + 1, s.J + (a + 1) * ld + bcol, bcol - a);
+      s.J[a * ld + bcol] = (((a == bcol) ? 1.0 : 0.0) - sum) * s.lam[a];
     }
   }
   c.sync();
   for (int idx = c.tid; idx < r * r; idx += c.nt) {
-    const int a = idx / r, bcol = idx - a * r;
+    const int a = fast_div(idx, s.div_r), bcol = idx - a * r;
     if (bcol >= a) {
-      const int pa = (int)s.wused[a];
+      const int pa = s.piv[a];
       s.Aacc[pa * ld + bcol] = s.dinv[pa] * s.J[a * ld + bcol];
     }
   }
-  // ---- P = F: scale column i of R back by ||g_i||
-  for (int idx = c.tid; idx < r * p; idx += c.nt) {
-    const int k = idx / p, i = idx - k * p;
-    s.P[k * ld + i] = (s.dinv[i] != 0.0) ? s.P[k * ld + i] / s.dinv[i] : 0.0;
-  }
-  c.sync();
-  int sw = 0;
+  // ---- P = F: scale column i of R back by ||g_i||; fn = ||f_i||^2
   for (int i = c.tid; i < p; i += c.nt) {
+    const double nrm = s.fn[i];
     double acc = 0.0;
-    for (int k = 0; k < r; ++k) { double v = s.P[k * ld + i]; acc += v * v; }
+    for (int k = 0; k < r; ++k) { const double v = s.P[k * ld + i] * nrm; s.P[k * ld + i] = v; acc = fma(v, v, acc); }
     s.fn[i] = acc;
   }
+  for (int idx = c.tid; idx < pp * ld; idx += c.nt) s.M[idx] = 0.0;     // M held the gathered columns
   c.sync();
+  int sw = 0;
 
+  s.div_r = make_div(r); s.div_p = make_div(p);
+  s.div_tr = make_div((r + 7) >> 3); s.div_tp = make_div((p + 7) >> 3);
   const bool grouped = nw > 0;
   const int workers = grouped ? nw : p;
   if (grouped) {
@@ -931,8 +1299,8 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
   }
   if (start == 0) {
-    if (grouped) (void)weights_and_objective_grouped(c, s, s.P, 0, r, p, coef, true, a);
-    else (void)weights_and_objective(c, s, s.P, 0, r, p, coef, true, a, cb, ca);
+    if (grouped) (void)weights_and_objective_grouped<LD>(c, s, s.P, 0, r, p, coef, true, a);
+    else (void)weights_and_objective<LD>(c, s, s.P, 0, r, p, coef, true, a, cb, ca);
   } else {
     // C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
     for (int idx = c.tid; idx < m * p; idx += c.nt) {
@@ -949,72 +1317,71 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       s.tmp[k * ld + i] = acc;
     }
     c.sync();
-    if (grouped) (void)weights_and_objective_grouped(c, s, s.tmp, 0, r, p, coef, false, a);
-    else (void)weights_and_objective(c, s, s.tmp, 0, r, p, coef, false, a, cb, ca);
+    if (grouped) (void)weights_and_objective_grouped<LD>(c, s, s.tmp, 0, r, p, coef, false, a);
+    else (void)weights_and_objective<LD>(c, s, s.tmp, 0, r, p, coef, false, a, cb, ca);
   }
 
   int m_eff = 0, rounds = iters;
   double prev_obj = 0.0;
   for (int t = 0; t < iters; ++t) {
+    sw = 0;
     for (int i = c.tid; i < p; i += c.nt) s.wused[i] = s.w[i];
     if (grouped) for (int i = c.tid; i < nw; i += c.nt) s.gwused[i] = s.gw[i];
-    // ---- T = P M P^T (current basis)
+    // ---- T = P M P^T (current basis); only one triangle is taken from the product, so that T is
+    // symmetric to the last bit
     if (coef > 0.0) {
-      for (int idx = c.tid; idx < p * r; idx += c.nt) {       // tmp[i][a] = sum_j M[i][j] P[a][j]
-        int i = idx / r, a = idx - i * r;
-        double acc = 0.0;
-        for (int j = 0; j < p; ++j) acc += s.M[i * ld + j] * s.P[a * ld + j];
-        s.tmp[i * ld + a] = acc;
+      matmul<LD, 1, 1, LD>(c, p, r, p, s.div_tr, s.M, s.P, [&](int i, int a, double v) { s.tmp[i * ld + a] = v; });   // tmp = M P^T
+      c.sync();
+      matmul<LD, 1, LD, 1>(c, r, r, p, s.div_tr, s.P, s.tmp,
+                           [&](int a, int b, double v) { if (a <= b) { s.T[a * ld + b] = v; s.T[b * ld + a] = v; } });
+    } else {
+      for (int idx = c.tid; idx < r * p; idx += c.nt) {                                   // tmp = P diag(w)
+        const int a = fast_div(idx, s.div_p), i = idx - a * p;
+        s.tmp[a * ld + i] = s.w[i] * s.P[a * ld + i];
       }
       c.sync();
-      for (int idx = c.tid; idx < r * r; idx += c.nt) {
-        int a = idx / r, b = idx - a * r;
-        if (b < a) continue;
-        double acc = 0.0;
-        for (int i = 0; i < p; ++i) acc += s.P[a * ld + i] * s.tmp[i * ld + b];
-        s.T[a * ld + b] = acc; s.T[b * ld + a] = acc;
-      }
-    } else {
-      for (int idx = c.tid; idx < r * r; idx += c.nt) {
-        int a = idx / r, b = idx - a * r;
-        if (b < a) continue;
-        double acc = 0.0;
-        for (int i = 0; i < p; ++i) acc += s.w[i] * s.P[a * ld + i] * s.P[b * ld + i];
-        s.T[a * ld + b] = acc; s.T[b * ld + a] = acc;
-      }
-    }
-    for (int idx = c.tid; idx < pp * pp; idx += c.nt) {
-      int a = idx / pp, b = idx - a * pp;
-      s.J[a * ld + b] = (a == b) ? 1.0 : 0.0;
-      if (a >= r || b >= r) s.T[a * ld + b] = 0.0;
+      matmul<LD, 1, 1, LD>(c, r, r, p, s.div_tr, s.tmp, s.P,
+                           [&](int a, int b, double v) { if (a <= b) { s.T[a * ld + b] = v; s.T[b * ld + a] = v; } });
     }
     c.sync();
-    sw = jacobi<LARGE>(c, s, &s.T, &s.tmp, &s.J, &s.M, r, r);   // M is free until the next weights
-    if (sw >= kMaxSweeps) status |= ST_EIG_SWEEPS;
-    m_eff = sort_eigs(c, s, s.T, r, m);
+    // ---- eigenvectors of T.  From the second round on T is close to diagonal here (the basis is the
+    // previous round's eigenbasis), the closer the further the rounds have converged: the refinement
+    // is tried first, and each time it declines one Jacobi sweep is made, the coordinates are taken
+    // to the swept basis and T is looked at again.
+    for (;;) {
+      if (refine_eig<LD>(c, s, r)) break;
+      const int ppr = (r + 1) & ~1;                       // the sweeps work on an even number of indices
+      for (int idx = c.tid; idx < ppr * ld; idx += c.nt) s.J[idx] = 0.0;
+      if (ppr > r) for (int b = c.tid; b < ppr; b += c.nt) { s.T[r * ld + b] = 0.0; s.T[b * ld + r] = 0.0; }
+      c.sync();
+      for (int a = c.tid; a < ppr; a += c.nt) s.J[a * (ld + 1)] = 1.0;
+      c.sync();
+      int big = 0;
+      sw += jacobi<LD>(c, s, &s.T, &s.tmp, &s.J, &s.M, r, r, 1, &big);   // M is free until the next weights
+      const bool last = !big || sw >= kMaxSweeps;
+      if (big && last) status |= ST_EIG_SWEEPS;
+      if (last) break;           // diagonal to rounding level (or given up): J holds the eigenvectors
+      matmul<1, LD, LD, 1>(c, r, p, r, s.div_tp, s.J, s.P, [&](int k, int i, double v) { s.tmp[k * ld + i] = v; });   // P <- J^T P
+      matmul<LD, 1, LD, 1>(c, p, r, r, s.div_tr, s.Aacc, s.J, [&](int i, int k, double v) { s.M[i * ld + k] = v; },
+                           ((r + 7) >> 3) * ((p + 7) >> 3));                                                        // Aacc <- Aacc J
+      c.sync();
+      { double* x = s.P; s.P = s.tmp; s.tmp = x; }
+      { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
+    }
+    s.count_sweeps += sw;
+    m_eff = sort_eigs<LD>(c, s, s.T, r, m);
 
     // ---- rotate into the new (sorted) eigenbasis: P <- J^T P, Aacc <- Aacc J
-    for (int idx = c.tid; idx < r * p; idx += c.nt) {
-      int k = idx / p, i = idx - k * p;
-      int col = s.ord[k];
-      double acc = 0.0;
-      for (int l = 0; l < r; ++l) acc += s.J[l * ld + col] * s.P[l * ld + i];
-      s.tmp[k * ld + i] = acc;
-    }
-    for (int idx = c.tid; idx < p * r; idx += c.nt) {
-      int i = idx / r, k = idx - i * r;
-      int col = s.ord[k];
-      double acc = 0.0;
-      for (int l = 0; l < r; ++l) acc += s.Aacc[i * ld + l] * s.J[l * ld + col];
-      s.M[i * ld + k] = acc;
-    }
+    matmul<1, LD, LD, 1>(c, r, p, r, s.div_tp, s.J, s.P, [&](int k, int i, double v) { s.tmp[k * ld + i] = v; }, 0, s.ord, nullptr);
+    matmul<LD, 1, LD, 1>(c, p, r, r, s.div_tr, s.Aacc, s.J, [&](int i, int k, double v) { s.M[i * ld + k] = v; },
+                         ((r + 7) >> 3) * ((p + 7) >> 3), nullptr, s.ord);
     c.sync();
     { double* x = s.P; s.P = s.tmp; s.tmp = x; }
     { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
 
     // ---- terms of Eq. (5) at the new subspace, and the next round's weights
-    double obj = grouped ? weights_and_objective_grouped(c, s, s.P, m_eff, r, p, coef, false, a)
-                         : weights_and_objective(c, s, s.P, m_eff, r, p, coef, false, a, cb, ca);
+    double obj = grouped ? weights_and_objective_grouped<LD>(c, s, s.P, m_eff, r, p, coef, false, a)
+                         : weights_and_objective<LD>(c, s, s.P, m_eff, r, p, coef, false, a, cb, ca);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
     if (tol >= 0.0 && t >= 1 && fabs(prev_obj - obj) <= tol) {      // same value in every thread
       rounds = t + 1;
