@@ -1,15 +1,21 @@
 """The five workloads at their full sizes, in the launch configuration bench.py times.
 
-cfg1 and cfg2 (the headline workload) are compared with a full run of the CPU oracle.  For cfg3,
-cfg4 and cfg5 a full n-space oracle run does not fit the time / memory of a test, so the result is
-pinned through quantities the oracle can compute at that size and properties that hold at any
-size:
+cfg1 and cfg2 (the headline workload) are compared with a full run of the CPU oracle inside the
+test.  For the larger workloads the oracle's full-size run takes from half an hour to hours (its
+column-blocked mode, fa_aggregate_blocked), so it was made once by
+tests/golden/make_fullsize_goldens.py and its p-dimensional results are stored in
+tests/golden/<workload>_full.npz: inner products, Eq. (5) per round, the last weights, the
+coordinates Z = G Y of every gradient in the oracle's subspace, the aggregate at about 8200 seeded
+columns and its norm.  The whole CUDA path is compared with those.  A workload without a stored run
+falls back to quantities the oracle can compute at that size and properties that hold at any size:
   * K against the oracle's plain inner products (accumulated over column blocks);
   * the subspace from the full path against the IRLS kernel fed with the oracle's K (that kernel
     is compared with the oracle round by round in test_gpu_parity.py);
   * Y orthonormal: A^T K A = I with the oracle's K;
   * sampled outputs: out[j] = (1/p) * sum_i (A A^T K 1)_i G[i][j], evaluated in fp64 one by one.
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -61,8 +67,84 @@ def test_full_size_matches_a_full_oracle_run(fa, name):
     assert rel < TOL[w.dtype][0] and ang < TOL[w.dtype][1]
 
 
+def _golden(name):
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", f"{name}_full.npz")
+    return np.load(path) if os.path.exists(path) else None
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5"])
+def test_full_size_matches_the_stored_oracle_run(fa, name):
+    gold = _golden(name)
+    if gold is None:
+        pytest.skip(f"no stored full-size oracle run for {name} (see test_full_size_properties)")
+    w = si.WORKLOADS[name]
+    assert (int(gold["n"]), int(gold["p"]), int(gold["m"]), float(gold["lam"]), int(gold["iters"]), int(gold["seed"])) == \
+           (w.n, w.p, w.m, w.lam, w.iters, w.seed)
+    G = _upload(si.generate(w))
+    p, n, m = w.p, w.n, w.m
+    A = torch.zeros((p, m), dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = fa.fa_aggregate(G, m, w.lam, w.iters, A_out=A, status=status)
+    K = fa.fa_gram(G)
+    obj = torch.zeros(w.iters, dtype=torch.float64, device="cuda")
+    wts = torch.zeros(p, dtype=torch.float64, device="cuda")
+    fa.fa_irls(K, m, w.lam, w.iters, w_out=wts, obj_out=obj)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rel_tol, ang_tol = TOL[w.dtype]
+    tensor_cores = w.dtype == "bf16" and p > 16
+
+    # inner products against the oracle's
+    Kref = gold["K"]
+    scale = np.sqrt(np.outer(np.diag(Kref), np.diag(Kref)))
+    gram_err = float(np.max(np.abs(K.cpu().numpy() - Kref) / scale))
+    assert gram_err < (2e-6 if tensor_cores else 5e-7)
+
+    # subspace: principal angles between the oracle's Y and Y_g = G^T A from p-dimensional quantities.
+    # Y^T Y_g = Z^T A (Z = G Y), Y_g^T Y_g = A^T K A =: W = L L^T with the oracle's K, so the squared
+    # sines are the eigenvalues of L^-1 (W - A^T Z Z^T A) L^-T.
+    k = int(gold["k"])
+    Ah = A.cpu().numpy()
+    assert k == m and not np.isnan(Ah).any()
+    Z = gold["Z"]
+    W = Ah.T @ Kref @ Ah
+    orth = float(np.abs(W - np.eye(m)).max())
+    assert orth < (2e-5 if tensor_cores else 1e-6)       # orthonormal in the GPU's own K; off by the error of K
+    Linv = np.linalg.inv(np.linalg.cholesky(W))
+    C = Ah.T @ Z
+    sin2 = np.linalg.eigvalsh(Linv @ (W - C @ C.T) @ Linv.T)
+    ang = float(np.arcsin(np.sqrt(np.clip(sin2.max(), 0.0, 1.0))))
+    assert ang < ang_tol, f"principal angle {ang}"
+
+    # Eq. (5) per round and the last weights, from the GPU's own inner products.  In the first rounds
+    # the cut between kept and discarded directions runs through a cluster of nearly equal eigenvalues
+    # (relative gaps of 1e-4 at these n), which amplifies the 1e-9 error of the inner products: the two
+    # trajectories part by up to a few 1e-3 in the objective around rounds 4-7 and meet again (1e-7 at
+    # the last round at p = 31).  So: a loose bound on every round, a tight one on where the rounds end.
+    diff = np.abs(obj.cpu().numpy() - gold["objective"])
+    w_err = float(np.max(np.abs(wts.cpu().numpy() - gold["w"]) / np.maximum(np.abs(gold["w"]), 1e-300)))
+    print(f"{name}: objective differences per round {diff}")
+    obj_err = float(diff[-1])
+    assert diff.max() < 2e-2 and obj_err < 1e-5 and w_err < 1e-2
+
+    # the aggregate at the stored columns (relative L2 over the sample, and element by element
+    # against the root-mean-square entry), and its norm
+    idx = gold["idx"]
+    got = out[torch.from_numpy(idx).cuda()].cpu().numpy().astype(np.float64)
+    ref = gold["d_sample"]
+    rel = fo.rel_l2(got, ref)
+    rms = float(gold["d_norm"]) / np.sqrt(n)
+    worst = float(np.max(np.abs(got - ref))) / rms
+    norm_err = abs(float(torch.linalg.vector_norm(out.double()).item()) - float(gold["d_norm"])) / float(gold["d_norm"])
+    print(f"{name}: gram_err={gram_err:.2e} orth={orth:.2e} angle={ang:.2e} obj_err={obj_err:.2e} w_err={w_err:.2e} "
+          f"rel_l2(sample)={rel:.2e} worst/rms={worst:.2e} norm_err={norm_err:.2e}")
+    assert rel < rel_tol and worst < 10 * rel_tol and norm_err < rel_tol
+
+
 @pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5"])
 def test_full_size_properties(fa, name):
+    if _golden(name) is not None:
+        pytest.skip("compared with the stored full-size oracle run instead")
     w = si.WORKLOADS[name]
     G_np = si.generate(w)
     G = _upload(G_np)

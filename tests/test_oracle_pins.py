@@ -646,3 +646,31 @@ def test_blocked_iteration_widens_the_stored_type_block_by_block():
     a = fo.fa_aggregate_blocked(G32, 3, 0.1, 3, block=100, widen=widen)
     b = fo.fa_aggregate(G32.astype(np.float64), 3, 0.1, 3)
     assert max(calls) == 100 and fo.rel_l2(a["d"], b["d"]) < 1e-10
+
+
+# ---- the stored full-size oracle runs (tests/golden/*_full.npz) are self-consistent ----------------------
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg4", "cfg5"])
+def test_stored_full_size_runs_are_self_consistent(name):
+    import os
+    import synthetic_inputs as si
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", f"{name}_full.npz")
+    if not os.path.exists(path):
+        pytest.skip(f"no stored run for {name}")
+    g = np.load(path)
+    w = si.WORKLOADS[name]
+    assert (int(g["n"]), int(g["p"]), int(g["m"]), float(g["lam"]), int(g["iters"]), int(g["seed"])) == \
+           (w.n, w.p, w.m, w.lam, w.iters, w.seed)
+    K, Z, u = g["K"], g["Z"], g["u"]
+    assert g["yty_err"] < 1e-10 and np.allclose(K, K.T, rtol=1e-13)
+    # u_i was summed from residual vectors; Z_i = Y^T g_i gives the same value as 1 - |Z_i|^2 / |g_i|^2 (Section 2.1)
+    nz = np.diag(K) > 0
+    assert np.allclose(u[nz], 1.0 - (Z[nz] ** 2).sum(axis=1) / np.diag(K)[nz], rtol=0, atol=1e-9)
+    # D2 from difference vectors against the inner products
+    D2 = np.diag(K)[:, None] + np.diag(K)[None, :] - 2 * K
+    assert np.allclose(g["D2"], D2, rtol=1e-9, atol=1e-9 * np.diag(K).max())
+    # the iteration descends from round two on (majorisation), and the aggregate is no longer than the plain mean's bound
+    obj = g["objective"]
+    assert all(obj[t + 1] <= obj[t] + 1e-9 for t in range(1, len(obj) - 1))
+    assert g["d_norm"] <= np.sqrt(K.sum()) / w.p * (1 + 1e-12)        # |Y Y^T mean| <= |mean|
+    assert len(g["idx"]) == len(g["d_sample"]) and g["idx"].max() == w.n - 1
