@@ -93,6 +93,84 @@ __global__ void __launch_bounds__(kThreads) combine_kernel(const T* __restrict__
   }
 }
 
+// fp32 rows that start on 8-byte but not all on 16-byte boundaries (n even with n % 4 = 2, or a base
+// that is 8 modulo 16): every row is still read with 16-byte loads.  A thread owns columns 4g..4g+3.
+// From a row whose start is 8 modulo 16 ("shifted") it loads the aligned vector at columns
+// 4g-2..4g+1: the upper half belongs to its own columns 0 and 1, the lower half to columns 2 and 3
+// of the thread that owns the group before (g - 1), for which it keeps a second pair of sums.  At
+// the end the pair is handed over with one shuffle.  Groups are walked from the end of the rows
+// backwards (see the kernel above), so group g - 1 sits in the next lane; the first lane of a warp
+// has no lane to receive from and reads its columns 2 and 3 of the shifted rows itself (8-byte
+// loads, 1/32 of the threads).  The thread of group 0 must not read before the matrix, and the last
+// two columns (n % 4 = 2) form a half group: both use 8-byte loads where a vector would leave the row.
+__global__ void __launch_bounds__(kThreads) combine_shifted_kernel(const float* __restrict__ G, int p, long long n,
+                                                                  const float* __restrict__ c, float* __restrict__ out,
+                                                                  int shift0, int nmod) {
+  __shared__ float cs[64];
+  float mine = 0.f;
+  if (threadIdx.x < 64) { mine = threadIdx.x < p ? c[threadIdx.x] : 0.f; cs[threadIdx.x] = mine; }
+  const int any = __syncthreads_or(mine != 0.f);
+  const long long full = n / 4;                         // whole groups; a half group of two columns may follow
+  const long long groups = full + ((n & 3) ? 1 : 0);
+  const long long g = groups - 1 - ((long long)blockIdx.x * kThreads + threadIdx.x);
+  const bool live = g >= 0;
+  const bool half = live && g == full;                  // the two columns n-2, n-1
+  const long long col = (live ? g : 0) * 4;
+  if (!any) {   // c = 0 (rejected or all-zero input): the result is exactly zero whatever G holds
+    if (live) for (int e = 0; e < (half ? 2 : 4); ++e) out[col + e] = 0.f;
+    return;
+  }
+  const int lane = threadIdx.x & 31;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;         // own columns
+  float b0 = 0.f, b1 = 0.f;                             // columns 2, 3 of group g - 1, from shifted rows
+  float e0 = 0.f, e1 = 0.f;                             // own columns 2, 3 from shifted rows, first lane only
+  if (live) {
+    for (int i0 = 0; i0 < p; i0 += 8) {
+      float4 v[8];
+      float2 w[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = i0 + k;
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        w[k] = make_float2(0.f, 0.f);
+        if (i < p) {
+          const float* row = G + (size_t)i * n + col;
+          const bool shifted = ((shift0 + i * nmod) & 3) != 0;
+          if (!shifted) {
+            if (!half) v[k] = __ldcs(reinterpret_cast<const float4*>(row));
+            else { const float2 t = __ldcs(reinterpret_cast<const float2*>(row)); v[k].x = t.x; v[k].y = t.y; }
+          } else {
+            if (g > 0) v[k] = __ldcs(reinterpret_cast<const float4*>(row - 2));            // columns 4g-2 .. 4g+1
+            else { const float2 t = __ldcs(reinterpret_cast<const float2*>(row)); v[k].z = t.x; v[k].w = t.y; }
+            if (lane == 0 && !half) w[k] = __ldcs(reinterpret_cast<const float2*>(row + 2));
+          }
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int i = i0 + k;
+        const float ck = i < p ? cs[i] : 0.f;
+        const bool shifted = ((shift0 + i * nmod) & 3) != 0;
+        if (!shifted) {
+          a0 = fmaf(ck, v[k].x, a0); a1 = fmaf(ck, v[k].y, a1); a2 = fmaf(ck, v[k].z, a2); a3 = fmaf(ck, v[k].w, a3);
+        } else {
+          b0 = fmaf(ck, v[k].x, b0); b1 = fmaf(ck, v[k].y, b1); a0 = fmaf(ck, v[k].z, a0); a1 = fmaf(ck, v[k].w, a1);
+          e0 = fmaf(ck, w[k].x, e0); e1 = fmaf(ck, w[k].y, e1);
+        }
+      }
+    }
+  }
+  // columns 2, 3 of this group from the shifted rows: summed by the thread of group g + 1 (previous lane)
+  const float r0 = __shfl_up_sync(0xffffffffu, b0, 1), r1 = __shfl_up_sync(0xffffffffu, b1, 1);
+  if (!live) return;
+  a2 += (lane == 0) ? e0 : r0;
+  a3 += (lane == 0) ? e1 : r1;
+  float* o = out + col;
+  if (half) { __stcs(o, a0); __stcs(o + 1, a1); return; }
+  if ((reinterpret_cast<uintptr_t>(o) % 16) == 0) __stcs(reinterpret_cast<float4*>(o), make_float4(a0, a1, a2, a3));
+  else { __stcs(o, a0); __stcs(o + 1, a1); __stcs(o + 2, a2); __stcs(o + 3, a3); }
+}
+
 template <typename T, int V>
 static cudaError_t run(const void* G, int p, long long n, const float* c, float* out, cudaStream_t st) {
   const long long groups = n / V;
@@ -108,6 +186,13 @@ cudaError_t launch_combine(const void* G, int dtype, int p, long long n, const f
   const uintptr_t a = reinterpret_cast<uintptr_t>(G);
   if (dtype == 0) {
     if (n % 4 == 0 && a % 16 == 0) return combine::run<float, 4>(G, p, n, c, out, st);
+    if (n % 2 == 0 && a % 8 == 0 && n >= 8) {            // every row on an 8-byte boundary: 16-byte loads with a hand-over
+      const long long groups = n / 4 + ((n & 3) ? 1 : 0);
+      const long long blocks = (groups + combine::kThreads - 1) / combine::kThreads;
+      combine::combine_shifted_kernel<<<(unsigned)blocks, combine::kThreads, 0, st>>>(
+          static_cast<const float*>(G), p, n, c, out, (int)((a % 16) / 4), (int)(n % 4));
+      return cudaGetLastError();
+    }
     if (n % 2 == 0 && a % 8 == 0) return combine::run<float, 2>(G, p, n, c, out, st);
     return combine::run<float, 1>(G, p, n, c, out, st);
   }

@@ -47,6 +47,10 @@ LADDER = [
     # fp32, 16 < p <= 32, rows on 16-byte boundaries: the tensor-fed kernel with teams of four warps
     (31, 50_000, "dup_zero", False, 0), (17, 4_096, "gauss", False, 0), (32, 300_004, "noisy_mean", False, 0),
     (24, 1_000_000, "gauss", False, 4), (31, 4_100, "noisy_mean", False, 0),
+    # fp32 rows on 8-byte but not all on 16-byte boundaries (n % 4 = 2 and / or a base that is 8 modulo 16):
+    # the output pass reads 16-byte vectors and hands half of them to the neighbouring thread
+    (15, 65_538, "noisy_mean", False, 2), (16, 10, "gauss", False, 0), (3, 8, "gauss", False, 2),
+    (9, 130, "noisy_mean", False, 0), (33, 4_098, "dup_zero", False, 2), (64, 1_026, "gauss", False, 0),
     # bf16, p > 16, 16-byte aligned rows: the tensor-core kernel
     (17, 64, "gauss", True, 0), (33, 264, "noisy_mean", True, 0), (63, 4_096, "dup_zero", True, 0),
     (64, 65_536, "gauss", True, 0), (31, 1_000_000, "dup_zero", True, 8), (48, 300_008, "noisy_mean", True, 0),
