@@ -107,6 +107,24 @@ def test_reference_arm_prints_one_json_line():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0
+    # same config keys as the GPU arm's line, and the extrapolation is declared
+    sys.path.insert(0, ROOT)
+    import bench
+    import synthetic_inputs as si
+    assert set(line["config"]) == set(bench.workload_config(si.WORKLOADS["cfg1"], 65_536, 3, "single GPU"))
+    assert line["steps_run"] == 1 and 0 < line["extrapolated_from_n"] <= 65_536
+
+
+def test_which_step_the_gpu_count_selects():
+    """`--gpus N` alone must time the n-sharded step (one job over N GPUs); replicas and the
+    worker-resident variant are opt-in; one GPU has a single mode whatever the flags."""
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.multi_gpu_mode(1, False, False) == "single"
+    assert bench.multi_gpu_mode(1, True, True) == "single"
+    assert bench.multi_gpu_mode(2, False, False) == "sharded"
+    assert bench.multi_gpu_mode(8, False, True) == "worker-resident"
+    assert bench.multi_gpu_mode(8, True, False) == "replicas"
 
 
 def _rank_main(rank, world, port, q):
