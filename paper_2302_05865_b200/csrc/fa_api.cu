@@ -3,21 +3,23 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/fa.h"
 #include "fa_kernels.h"
 
 namespace fa {
 
 int sm_count() {
-  static int cached[64];
+  static std::atomic<int> cached[64];                  // zero-initialised; a slot is published once, whole
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
-  if (cached[dev] == 0) {
-    int v = 0;
+  int v = cached[dev].load(std::memory_order_acquire);
+  if (v == 0) {
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-    cached[dev] = v;
+    cached[dev].store(v, std::memory_order_release);   // concurrent first calls store the same value
   }
-  return cached[dev];
+  return v;
 }
 
 namespace {

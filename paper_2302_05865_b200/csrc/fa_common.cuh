@@ -39,13 +39,37 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking test of a phase (try_wait above may suspend the thread for a system-dependent time).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+constexpr long long kShortWaitCycles = 1000000;      // limits below this poll without suspending
+
 // Wait for a phase with a cycle limit.  Returns false when the limit ran out (the caller then
-// records FA_ST_TIMEOUT and winds down); never spins unbounded.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// records FA_ST_TIMEOUT and winds down); never spins unbounded.  `limit` is the caller's primary
+// limit (a launch parameter where a test shortens it); waits that only let copies already in
+// flight land before a block exits always use the long default.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles) {
+  if (limit < kShortWaitCycles) {      // a deliberately short limit: the suspending form could outlast it
+    const long long t0 = clock64();
+    do {
+      if (mbar_test_wait(bar, parity)) return true;
+    } while (clock64() - t0 <= limit);
+    return false;
+  }
   if (mbar_try_wait(bar, parity)) return true;
   long long t0 = clock64();
   while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) return false;
+    if (clock64() - t0 > limit) return false;
   }
   return true;
 }
@@ -62,6 +86,33 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 
 __device__ __forceinline__ void fence_proxy_async() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Butterfly reduce-scatter of NACCP values per lane across the warp: afterwards lane l holds the
+// warp sums of elements [l*NACCP/32, (l+1)*NACCP/32) in x[0 .. NACCP/32).  NACCP is a multiple of 32.
+template <int NACCP, int L, int MASK>
+__device__ __forceinline__ void butterfly_step(float (&x)[NACCP], int lane) {
+  if constexpr (MASK >= 1) {
+    constexpr int H = L / 2;
+    const bool up = (lane & MASK) != 0;
+#pragma unroll
+    for (int k = 0; k < H; ++k) {
+      float lo = x[k], hi = x[H + k];
+      float send = up ? lo : hi;
+      float keep = up ? hi : lo;
+      x[k] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
+    }
+    butterfly_step<NACCP, H, MASK / 2>(x, lane);
+  }
+}
+
+template <int NACCP>
+__device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP / 32], int lane) {
+  butterfly_step<NACCP, NACCP, 16>(acc, lane);
+#pragma unroll
+  for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
+#pragma unroll
+  for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
 }
 
 // ---- element access: V consecutive elements at a V-element-aligned shared address -> floats

@@ -36,33 +36,6 @@ struct Params {
   int* status;
 };
 
-// Butterfly reduce-scatter of NACCP values per lane across the warp: afterwards lane l holds the
-// warp sums of elements [l*NACCP/32, (l+1)*NACCP/32) in x[0 .. NACCP/32).  NACCP is a multiple of 32.
-template <int NACCP, int L, int MASK>
-__device__ __forceinline__ void butterfly_step(float (&x)[NACCP], int lane) {
-  if constexpr (MASK >= 1) {
-    constexpr int H = L / 2;
-    const bool up = (lane & MASK) != 0;
-#pragma unroll
-    for (int k = 0; k < H; ++k) {
-      float lo = x[k], hi = x[H + k];
-      float send = up ? lo : hi;
-      float keep = up ? hi : lo;
-      x[k] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
-    }
-    butterfly_step<NACCP, H, MASK / 2>(x, lane);
-  }
-}
-
-template <int NACCP>
-__device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP / 32], int lane) {
-  butterfly_step<NACCP, NACCP, 16>(acc, lane);
-#pragma unroll
-  for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
-#pragma unroll
-  for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
-}
-
 struct Ring {
   uint64_t* full;
   uint64_t* empty;

@@ -23,6 +23,7 @@
 #include <cuda_bf16.h>
 
 #include "fa_common.cuh"
+#include "fa_tensor_map.cuh"
 #include "fa_gram_finish.cuh"
 #include "fa_kernels.h"
 
@@ -40,20 +41,14 @@ constexpr int kFold = 8;                        // runs added in fp32 registers 
 constexpr int kLoaderWarps = 4;                 // warps 6..9 fill the loader stages with cp.async copies
 constexpr int kMmaWarp2 = 6 + kLoaderWarps;       // second MMA issuer (odd tiles); warp 1 takes the even ones
 constexpr int kThreads = 192 + 32 * kLoaderWarps + 32;
-#ifndef FA_TC_ACCS
-#define FA_TC_ACCS 8
-#endif
-constexpr int kAccs = FA_TC_ACCS;               // 64-column accumulators in tensor memory, used in turn
+constexpr int kAccs = 8;               // 64-column accumulators in tensor memory, used in turn
 constexpr int kTmemCols = 64 * kAccs;
 static_assert(kAccs == 2 || kAccs == 4 || kAccs == 8, "tensor-memory allocations are powers of two");
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 64 * 64 * sizeof(double);
 
 // Stages whose bit is set in kLoaderMask are filled by the loader warps, the others by the
 // tensor-load thread; tile u goes to stage u mod kStages.
-#ifndef FA_TC_LOADER_MASK
-#define FA_TC_LOADER_MASK 0x2A
-#endif
-constexpr uint32_t kLoaderMask = FA_TC_LOADER_MASK;
+constexpr uint32_t kLoaderMask = 0x2A;
 constexpr int kLoaderDepth = ((kLoaderMask >> 0) & 1) + ((kLoaderMask >> 1) & 1) + ((kLoaderMask >> 2) & 1) +
                              ((kLoaderMask >> 3) & 1) + ((kLoaderMask >> 4) & 1) + ((kLoaderMask >> 5) & 1);
 static_assert(kLoaderDepth >= 1 && kLoaderDepth <= 3 && kLoaderMask < (1u << kStages), "loader stages");
@@ -83,14 +78,6 @@ constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          smem_u32(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
@@ -362,29 +349,6 @@ __global__ void __launch_bounds__(kThreads, 1) gram_tc_kernel(const __grid_const
 }  // namespace gramtc
 
 // ---- host side
-namespace {
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
-EncodeTiledFn encode_tiled() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-}  // namespace
-
 bool gram_tc_eligible(const void* G, int dtype, int p, long long n) {
   return dtype == 1 && p > 16 && p <= 64 && n % 8 == 0 && (reinterpret_cast<uintptr_t>(G) % 16) == 0 &&
          n < (1LL << 31) && encode_tiled() != nullptr;

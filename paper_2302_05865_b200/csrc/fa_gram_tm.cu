@@ -21,6 +21,8 @@
 // itself; every thread keeps the upper triangle for its columns, as in fa_gram.cu; products in
 // fp32, runs of at most 64 columns, warp butterfly into fp64.  Block totals and the last-block reduction are
 // the ones of fa_gram.cu (bit-reproducible, single launch).
+#include <atomic>
+
 #include "fa_gram_tm.cuh"
 #include "fa_gram_finish.cuh"
 #include "fa_kernels.h"
@@ -35,33 +37,8 @@ struct Params {
   unsigned int* counter;
   double* K;
   int* status;
+  long long wait_cycles;       // limit of a wait for a tile (kWaitCycles unless a test shortened it)
 };
-
-template <int NACCP, int L, int MASK>
-__device__ __forceinline__ void butterfly_step(float (&x)[NACCP], int lane) {
-  if constexpr (MASK >= 1) {
-    constexpr int H = L / 2;
-    const bool up = (lane & MASK) != 0;
-#pragma unroll
-    for (int k = 0; k < H; ++k) {
-      float lo = x[k], hi = x[H + k];
-      float send = up ? lo : hi;
-      float keep = up ? hi : lo;
-      x[k] = keep + __shfl_xor_sync(0xffffffffu, send, MASK);
-    }
-    butterfly_step<NACCP, H, MASK / 2>(x, lane);
-  }
-}
-
-// Reduce-scatter of NACCP values per lane over the warp, then into the lane's fp64 sums.
-template <int NACCP>
-__device__ __forceinline__ void flush(float (&acc)[NACCP], double (&dacc)[NACCP / 32], int lane) {
-  butterfly_step<NACCP, NACCP, 16>(acc, lane);
-#pragma unroll
-  for (int k = 0; k < NACCP / 32; ++k) dacc[k] += static_cast<double>(acc[k]);
-#pragma unroll
-  for (int k = 0; k < NACCP; ++k) acc[k] = 0.f;
-}
 
 // p <= 16.  No producer: every warp owns `depth` stages and keeps them loaded itself -- lane 0 issues
 // the tensor loads of the warp's next tile into the stage the warp has just finished with.  (One
@@ -83,10 +60,12 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
   double* totals = reinterpret_cast<double*>(smem + (size_t)kTriWarps * depth * stage_bytes);
   uint64_t* full = reinterpret_cast<uint64_t*>(totals + kTriWarps * NACCP);
   int* flag = reinterpret_cast<int*>(full + kTriWarps * kMaxDepth);      // last-block flag
+  int* aborted = flag + 1;                                               // a warp of this block gave up on a tile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
     for (int s = 0; s < kTriWarps * kMaxDepth; ++s) mbar_init(&full[s], 1);
+    *aborted = 0;
   }
   fence_proxy_async();
   __syncthreads();
@@ -130,15 +109,18 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
   int s = 0;
   uint32_t phase = 0;
   for (int t = tfirst; t < ntiles; t += tstride) {
-    if (!mbar_wait(&mybars[s], phase)) {
+    // the lanes poll on their own; once any of them has seen the phase complete, it is complete
+    if (!__any_sync(0xffffffffu, mbar_wait(&mybars[s], phase, prm.wait_cycles))) {
       if (lane == 0) {
         if (prm.status) atomicOr(prm.status, kStTimeout);
-        // let this warp's other loads land before the block can exit
+        *reinterpret_cast<volatile int*>(aborted) = 1;
+        // every load of this warp that is in flight -- the one it gave up on and those of the stages
+        // after it -- must land before the block can exit: these waits keep the long limit
         int s2 = s;
         uint32_t ph2 = phase;
-        for (int k = 1; k < depth; ++k) {
-          if (++s2 == depth) { s2 = 0; ph2 ^= 1u; }
+        for (int k = 0; k < depth; ++k) {
           if (t + k * tstride < ntiles) (void)mbar_wait(&mybars[s2], ph2);
+          if (++s2 == depth) { s2 = 0; ph2 ^= 1u; }
         }
       }
       break;
@@ -186,6 +168,9 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
     if (j < prm.p) {
       double sum = 0.0;
       for (int w = 0; w < kTriWarps; ++w) sum += totals[w * NACCP + e];
+      // a block that gave up has incomplete sums: NaN, so that K comes out non-finite and whoever
+      // reads it (the IRLS kernel sets FA_ST_NONFINITE and writes zeros) sees the failure
+      if (*reinterpret_cast<volatile int*>(aborted)) sum = __longlong_as_double(0x7ff8000000000000LL);
       prm.partials[(size_t)gram::canon_index(i, j, prm.p) * gridDim.x + blockIdx.x] = sum;
     }
   }
@@ -220,8 +205,10 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   double* totals = reinterpret_cast<double*>(smem + (size_t)2 * kQuadDepth * kStageBytes);
   uint64_t* full = reinterpret_cast<uint64_t*>(totals + kQuadWarps * kQuadAcc);
   int* flag = reinterpret_cast<int*>(full + 2 * kQuadDepth);
+  int* aborted = flag + 1;                   // [team]: a warp of the team gave up on a tile
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int team = warp >> 2, role = warp & 3;
+  if (tid == 0) { aborted[0] = 0; aborted[1] = 0; }
 
   for (int i = tid * 16; i < 2 * kQuadDepth * kStageBytes; i += kThreads * 16)
     *reinterpret_cast<uint4*>(stages + i) = make_uint4(0, 0, 0, 0);
@@ -259,48 +246,65 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   int s = 0;
   uint32_t phase = 0;
   for (int t = tfirst; t < ntiles; t += tstride) {
-    if (!mbar_wait(&mybars[s], phase)) {
-      if (lane == 0 && prm.status) atomicOr(prm.status, kStTimeout);
-      break;
+    // Giving up must be a decision of the whole team: its four warps meet at the team's barrier after
+    // every tile, so a warp whose wait ran out skips the tile, raises the team's flag and still goes
+    // to the barrier; behind it all four read the flag and leave together.
+    const bool ok = __any_sync(0xffffffffu, mbar_wait(&mybars[s], phase, prm.wait_cycles));
+    if (!ok && lane == 0) {
+      if (prm.status) atomicOr(prm.status, kStTimeout);
+      *reinterpret_cast<volatile int*>(&aborted[team]) = 1;
     }
-    const char* sbase = mystages + (size_t)s * kStageBytes;
-    if (role < 2) {
-#pragma unroll 1
-      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
-        const char* ptr = sbase + rowbase + cg * 8;
-        float x[16][2];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) SmemVec<float, 2>::load(ptr + i * kRowBytes, x[i]);
-        int idx = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-#pragma unroll
-          for (int j = i; j < 16; ++j) {
-            acc[idx] = fmaf(x[i][0], x[j][0], acc[idx]);
-            acc[idx] = fmaf(x[i][1], x[j][1], acc[idx]);
-            ++idx;
-          }
-      }
-    } else {
-#pragma unroll 1
-      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
-        const char* pa = sbase + rowbase + cg * 8;
-        const char* pb = sbase + 16 * kRowBytes + cg * 8;
-        float a[8][2], b[16][2];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) SmemVec<float, 2>::load(pa + i * kRowBytes, a[i]);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) SmemVec<float, 2>::load(pb + j * kRowBytes, b[j]);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
-            acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
-          }
+    if (ok) {
+      const char* sbase = mystages + (size_t)s * kStageBytes;
+      if (role < 2) {
+  #pragma unroll 1
+        for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+          const char* ptr = sbase + rowbase + cg * 8;
+          float x[16][2];
+  #pragma unroll
+          for (int i = 0; i < 16; ++i) SmemVec<float, 2>::load(ptr + i * kRowBytes, x[i]);
+          int idx = 0;
+  #pragma unroll
+          for (int i = 0; i < 16; ++i)
+  #pragma unroll
+            for (int j = i; j < 16; ++j) {
+              acc[idx] = fmaf(x[i][0], x[j][0], acc[idx]);
+              acc[idx] = fmaf(x[i][1], x[j][1], acc[idx]);
+              ++idx;
+            }
+        }
+      } else {
+  #pragma unroll 1
+        for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+          const char* pa = sbase + rowbase + cg * 8;
+          const char* pb = sbase + 16 * kRowBytes + cg * 8;
+          float a[8][2], b[16][2];
+  #pragma unroll
+          for (int i = 0; i < 8; ++i) SmemVec<float, 2>::load(pa + i * kRowBytes, a[i]);
+  #pragma unroll
+          for (int j = 0; j < 16; ++j) SmemVec<float, 2>::load(pb + j * kRowBytes, b[j]);
+  #pragma unroll
+          for (int i = 0; i < 8; ++i)
+  #pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
+              acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
+            }
+        }
       }
     }
     team_barrier(team);                  // all four parts are done with the stage
+    if (*reinterpret_cast<volatile int*>(&aborted[team])) {
+      if (issuer) {   // the team's loads in flight (this stage's and the following ones') must land: long limit
+        int s2 = s;
+        uint32_t ph2 = phase;
+        for (int k = 0; k < kQuadDepth; ++k) {
+          if (t + k * tstride < ntiles) (void)mbar_wait(&mybars[s2], ph2);
+          if (++s2 == kQuadDepth) { s2 = 0; ph2 ^= 1u; }
+        }
+      }
+      break;
+    }
     if (issuer) {
       fence_proxy_async();
       issue(t + kQuadDepth * tstride, s);
@@ -328,32 +332,15 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
       gi = 8 * (part - 2) + e / 16; gj = 16 + e % 16;
     }
     if (gi >= prm.p || gj >= prm.p) continue;
-    const double sum = totals[(size_t)part * kQuadAcc + e] + totals[(size_t)(4 + part) * kQuadAcc + e];
+    double sum = totals[(size_t)part * kQuadAcc + e] + totals[(size_t)(4 + part) * kQuadAcc + e];
+    if (*reinterpret_cast<volatile int*>(&aborted[0]) | *reinterpret_cast<volatile int*>(&aborted[1]))
+      sum = __longlong_as_double(0x7ff8000000000000LL);     // incomplete sums must not pass for inner products
     prm.partials[(size_t)gram::canon_index(gi, gj, prm.p) * gridDim.x + blockIdx.x] = sum;
   }
   gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
 }
 
 namespace {
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver's tensor-map encoder, looked up through the runtime (no link against libcuda).
-EncodeTiledFn encode_tiled() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
 
 // Row classes of a p x n matrix of S-byte elements: 0 when more than kMaxClasses would be needed.
 int class_count(long long n, int S) {
@@ -444,6 +431,23 @@ bool gram_tm32_eligible(const void* G, int dtype, int p, long long n) {
   return dtype == 0 && p > 16 && p <= 32 && gramtm::available(G, dtype, n) && (n % 4) == 0;
 }
 
+namespace {
+// Limit of the kernels' waits for a tile, in cycles.  Always kWaitCycles in normal use.
+std::atomic<long long> g_tile_wait_cycles{kWaitCycles};
+}  // namespace
+
+}  // namespace fa
+
+// Test hook (exported, but deliberately not declared in include/fa.h): shortens the tile waits of
+// the tensor-fed Gram kernels so that a test can watch a wait run out on a launch that is otherwise
+// correct -- the kernel gives up, lets its loads land (those waits keep the long limit), reports
+// FA_ST_TIMEOUT and returns.  cycles <= 0 restores the default.
+extern "C" void fa_test_set_gram_wait_cycles(long long cycles) {
+  fa::g_tile_wait_cycles.store(cycles > 0 ? cycles : fa::kWaitCycles);
+}
+
+namespace fa {
+
 cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
                              int* status, cudaStream_t st) {
   gramtm::Maps maps;
@@ -456,6 +460,7 @@ cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials
   prm.counter = counter;
   prm.K = K;
   prm.status = status;
+  prm.wait_cycles = g_tile_wait_cycles.load();
   const int sms = sm_count();
   const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
   cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
@@ -482,6 +487,7 @@ cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double*
   prm.counter = counter;
   prm.K = K;
   prm.status = status;
+  prm.wait_cycles = g_tile_wait_cycles.load();
   const int sms = sm_count();
   const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
   cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);

@@ -1,9 +1,7 @@
 // Shared between the Gram kernels that are fed by TMA tensor loads: the tensor maps of the row classes
 // and how a staged tile is laid out (see fa_gram_tm.cu for the scheme).
 #pragma once
-#include <cuda.h>
-
-#include "fa_common.cuh"
+#include "fa_tensor_map.cuh"
 
 namespace fa {
 namespace gramtm {
@@ -25,14 +23,6 @@ struct Layout {
   int rowbase[kMaxClasses];    // staged row index of the first row of class c
   int shift[kMaxClasses];      // elements between the map's row start and the row's own start
 };
-
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          smem_u32(dst)),
-      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
-}
 
 // Host: tensor maps and layout for a p x n matrix at G (16-byte aligned); false when the shape needs
 // more than kMaxClasses row classes or the driver's encoder is not available.

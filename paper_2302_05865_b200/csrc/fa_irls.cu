@@ -31,18 +31,11 @@ static cudaError_t launch_nt(const IrlsArgs& a, cudaStream_t st) {
 // One thread per Jacobi work item where the block size allows it: (p/2)^2 2x2 blocks plus
 // p * p/2 eigenvector row pairs.
 cudaError_t launch_irls(const IrlsArgs& a, cudaStream_t st) {
-#ifndef FA_IRLS_NT16
-#define FA_IRLS_NT16 256
-#endif
-#ifndef FA_IRLS_NT32
-#define FA_IRLS_NT32 512
-#endif
-#ifndef FA_IRLS_NT64
-#define FA_IRLS_NT64 512
-#endif
-  if (a.p <= 16) return launch_nt<FA_IRLS_NT16, 20>(a, st);
-  if (a.p <= 32) return launch_nt<FA_IRLS_NT32, 36>(a, st);
-  return launch_nt<FA_IRLS_NT64, 68>(a, st);
+  // 256 threads up to 16 gradients, 512 above: the matrix phases hand out 8 x 8 tiles to a power-of-two
+  // number of warps, and the Jacobi sweeps want one thread per work item where the block size allows it
+  if (a.p <= 16) return launch_nt<256, 20>(a, st);
+  if (a.p <= 32) return launch_nt<512, 36>(a, st);
+  return launch_nt<512, 68>(a, st);
 }
 
 }  // namespace fa

@@ -8,6 +8,8 @@
 // array exists once per GPU that loads the library and stays until the process exits.
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/fa.h"
 #include "fa_kernels.h"
 
@@ -20,16 +22,18 @@ static __device__ __align__(256) double g_gram_scratch[kScratchDoubles + 32];
 // Device address of the array, looked up once per device.  In host code `g_gram_scratch` is only a
 // handle for the runtime; the kernels need the address that cudaGetSymbolAddress returns.
 double* scratch_address(int* rc) {
-  static double* cached[64];
+  static std::atomic<double*> cached[64];              // per device; concurrent first calls look up the same address
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *rc = FA_ERR_CUDA; return nullptr; }
-  if (!cached[dev]) {
+  double* addr = cached[dev].load(std::memory_order_acquire);
+  if (!addr) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_gram_scratch) != cudaSuccess || !ptr) { *rc = FA_ERR_CUDA; return nullptr; }
-    cached[dev] = static_cast<double*>(ptr);
+    addr = static_cast<double*>(ptr);
+    cached[dev].store(addr, std::memory_order_release);
   }
   *rc = FA_OK;
-  return cached[dev];
+  return addr;
 }
 
 }  // namespace

@@ -105,3 +105,46 @@ def test_shard_bounds_are_aligned_and_cover():
             assert all(b[r][1] == b[r + 1][0] for r in range(world - 1))
             assert all(lo % sharded.SHARD_ALIGN == 0 or lo == n for lo, _ in b)
             assert max(hi - lo for lo, hi in b) == min(n, sharded.shard_size(n, world))
+
+
+def _rank_with_a_missing_peer(rank, world, port, q):
+    """Rank 1 never joins the all-reduce of the partial inner products; rank 0 must get an error from the
+    collective within its time limit instead of waiting for ever."""
+    import datetime
+    import time
+    import torch
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=datetime.timedelta(seconds=5))
+    sys.path.insert(0, ROOT)
+    from paper_2302_05865_b200 import sharded
+    if rank == 1:
+        time.sleep(12)                       # alive, but absent from the collective
+        q.put((rank, "absent"))
+        return
+    G = torch.from_numpy(_case(6, 64, 9))
+    lo, hi = sharded.shard_bounds(64, world, rank)
+    step = sharded.ShardedStep(3, 0.1, 4, ops=OracleOps)
+    t0 = time.time()
+    try:
+        step(G[:, lo:hi].contiguous())
+        q.put((rank, "returned"))
+    except Exception as e:                   # gloo reports the time-out as a RuntimeError
+        q.put((rank, f"error after {time.time() - t0:.1f} s: {type(e).__name__}"))
+
+
+def test_a_rank_missing_at_the_all_reduce_ends_the_collective_with_an_error():
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + (os.getpid() + 977) % 2000
+    procs = [ctx.Process(target=_rank_with_a_missing_peer, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = dict(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(30)
+        if p.is_alive():
+            p.kill()
+    assert got[0].startswith("error after"), got
+    assert float(got[0].split()[2]) < 11.0, got
