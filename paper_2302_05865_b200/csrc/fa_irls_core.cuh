@@ -66,6 +66,7 @@ constexpr int kMaxSweeps = 40;
 constexpr double kRefineTheta = 0.3;   // refinement is tried when every |T_ij| <= this * |T_jj - T_ii|
 constexpr double kRefineStop = 1e-8;   // ... and has converged when a step's largest correction is below this
 constexpr int kMaxRefine = 8;          // steps after which a refinement that has not converged is given up
+constexpr int kMaxSweepsF32 = 12;      // fp32 sweeps per round before the fp64 sweeps take over
 constexpr int kMaxP = 64;
 
 constexpr int ST_NONFINITE = 1, ST_RANK0 = 2, ST_RANK_LT_M = 4, ST_EIG_SWEEPS = 8;
@@ -120,7 +121,7 @@ struct Smem {
   int *grp, *first;
   int nw;
   int ld;
-  int count_sweeps, count_refinements;   // work done by the eigensolver in this call (diagnostics)
+  int count_sweeps, count_sweeps_f32, count_refinements;   // work done by the eigensolver in this call (diagnostics)
   FastDiv div_r, div_p, div_tr, div_tp;  // by the rank r, by p, by their numbers of 8-wide tiles
   int max_calls, sum_calls;              // block_max / block_sum calls so far (parity picks the exchange slots)
 };
@@ -155,7 +156,7 @@ FA_FN void carve(Smem& s, void* base, int p, int nt) {
   s.first = q; q += pp; s.piv = q; q += pp; s.flags = q; q += 8;
   s.pairs = reinterpret_cast<unsigned short*>(q);
   s.nw = 0;
-  s.count_sweeps = 0; s.count_refinements = 0;
+  s.count_sweeps = 0; s.count_sweeps_f32 = 0; s.count_refinements = 0;
   s.div_r = s.div_p = s.div_tr = s.div_tp = make_div(1);
   s.max_calls = 0; s.sum_calls = 0;
 }
@@ -406,9 +407,37 @@ FA_FN bool rotation_of(double app, double aqq, double apq, double& cs, double& s
   return ok && (m2 > (kJacobiBig * kJacobiBig) * ref2);
 }
 
-FA_FN bool rotation(const double* T, int ld, int a, int b, int dim, double& cs, double& sn) {
-  if (b >= dim) { cs = 1.0; sn = 0.0; return false; }
-  return rotation_of(T[a * ld + a], T[b * ld + b], T[a * ld + b], cs, sn);
+// The same rotation in fp32, for sweeps whose only job is to bring T close enough to diagonal form for
+// the fp64 refinement to take over (which also repairs the orthogonality the fp32 products lose): the
+// chain of dependent operations is less than half as long (fp32 FMA 4 cycles, hardware rsqrt).
+// Entries are expected scaled to order one.
+FA_FN bool rotation_of(float app, float aqq, float apq, float& cs, float& sn) {
+  constexpr float kTol = 3e-8f, kBig = 1e-3f;
+  const float m2 = apq * apq, ref2 = fabsf(app * aqq);
+  const bool ok = (m2 > (kTol * kTol) * ref2) && (m2 > 1e-30f);
+  const float d = aqq - app, h = 2.0f * apq;
+  const float q = fmaf(d, d, h * h);
+  const float qs = ok ? q : 1.0f;
+#ifndef FA_IRLS_HOST
+  const float rinv = rsqrtf(qs);
+#else
+  const float rinv = 1.0f / sqrtf(qs);
+#endif
+  const float hr = (0.5f * h) * rinv;
+  const float x = fmaf(0.5f * fabsf(d), rinv, 0.5f);           // cos^2 phi, in [1/2, 1]
+#ifndef FA_IRLS_HOST
+  const float cinv = rsqrtf(x);
+#else
+  const float cinv = 1.0f / sqrtf(x);
+#endif
+  float c = x * cinv, sv = hr * cinv;
+  const float e = fmaf(c, c, fmaf(sv, sv, -1.0f));
+  const float f = fmaf(e, -0.5f, 1.0f);
+  c *= f;
+  sv *= f;
+  cs = ok ? c : 1.0f;
+  sn = ok ? (d < 0.0f ? -sv : sv) : 0.0f;
+  return ok && (m2 > (kBig * kBig) * ref2);
 }
 
 // Systolic (Brent-Luk) arrangement of np pairs: pair k sits at positions (k, np + k) -- "top" entries
@@ -445,16 +474,16 @@ FA_FN int systolic_next(int x, int np) {
 // A full sweep (pp - 1 rounds) returns every index to its own position, and sweeps are never cut
 // short.  On return *Tio / *Jio point at the buffers that hold the results.  Returns the sweeps made.
 // Up to 8 pairs on the device; any size on the host.
-template <int LD>
-FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
+template <int LD, typename R>
+FA_FN int jacobi_small(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** Jaltio,
                        int dim, int jrows, int max_sweeps, int* big_out) {
   constexpr int ld = LD;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
-  double* T = *Tio;
-  double* Tn = *Taltio;
-  double* J = *Jio;
-  double* Jn = *Jaltio;
+  R* T = *Tio;
+  R* Tn = *Taltio;
+  R* J = *Jio;
+  R* Jn = *Jaltio;
   const int nb2 = np * np, total2 = nb2 + jrows * np;
   // the item this thread owns for the whole solve (element offsets into T / J)
   struct Item { int kind, diag, ksrc, kaa, kbb, kab, laa, lbb, lab, x0, x1, x2, x3, z0, z1, z2, z3; } it;
@@ -500,22 +529,22 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       {
         // every lane with an item works out the rotation of its column pair l; a block of T gets
         // its row rotation from the lane `ksrc` of its warp (worked out here only if there is none)
-        double cl = 1.0, sl = 0.0;
+        R cl = 1.0, sl = 0.0;
         bool bigl = false;
-        double xac = 0.0, xad = 0.0, xbc = 0.0, xbd = 0.0;
+        R xac = 0.0, xad = 0.0, xbc = 0.0, xbd = 0.0;
         if (it.kind != 0) {
-          const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+          const R laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
           if (it.kind == 1) { xac = T[it.x0]; xad = T[it.x1]; xbc = T[it.x2]; xbd = T[it.x3]; }
           else { xac = J[it.x0]; xad = J[it.x1]; }
           bigl = rotation_of(laa, lbb, lab, cl, sl);
         }
         const int src = it.ksrc < 0 ? 0 : it.ksrc;
-        double ck = __shfl_sync(0xffffffffu, cl, src), sk = __shfl_sync(0xffffffffu, sl, src);
+        R ck = __shfl_sync(0xffffffffu, cl, src), sk = __shfl_sync(0xffffffffu, sl, src);
         if (it.kind == 1) {
           if (it.ksrc < 0) (void)rotation_of(T[it.kaa], T[it.kbb], T[it.kab], ck, sk);
           if (it.diag && bigl) *big = 1;
-          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+          const R yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+          const R ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
           Tn[it.z0] = cl * yac - sl * yad; Tn[it.z1] = sl * yac + cl * yad;
           Tn[it.z2] = cl * ybc - sl * ybd; Tn[it.z3] = sl * ybc + cl * ybd;
         } else if (it.kind == 2) {
@@ -525,21 +554,21 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
       }
 #else
       if (it.kind == 1) {
-        const double kaa = T[it.kaa], kbb = T[it.kbb], kab = T[it.kab];
-        const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
-        const double xac = T[it.x0], xad = T[it.x1], xbc = T[it.x2], xbd = T[it.x3];
-        double ck, sk, cl, sl;
+        const R kaa = T[it.kaa], kbb = T[it.kbb], kab = T[it.kab];
+        const R laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+        const R xac = T[it.x0], xad = T[it.x1], xbc = T[it.x2], xbd = T[it.x3];
+        R ck, sk, cl, sl;
         const bool bigk = rotation_of(kaa, kbb, kab, ck, sk);
         (void)rotation_of(laa, lbb, lab, cl, sl);
         if (it.diag && bigk) *big = 1;
-        const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-        const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+        const R yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+        const R ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
         Tn[it.z0] = cl * yac - sl * yad; Tn[it.z1] = sl * yac + cl * yad;
         Tn[it.z2] = cl * ybc - sl * ybd; Tn[it.z3] = sl * ybc + cl * ybd;
       } else if (it.kind == 2) {
-        const double laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
-        const double va = J[it.x0], vb = J[it.x1];
-        double cl, sl;
+        const R laa = T[it.laa], lbb = T[it.lbb], lab = T[it.lab];
+        const R va = J[it.x0], vb = J[it.x1];
+        R cl, sl;
         (void)rotation_of(laa, lbb, lab, cl, sl);
         Jn[it.z0] = cl * va - sl * vb;
         Jn[it.z1] = sl * va + cl * vb;
@@ -550,15 +579,15 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
         if (idx < nb2) {
           const int k = idx / np, l = idx - k * np;
           const int a = k, b = np + k, cc = l, d = np + l;
-          const double kaa = T[a * ld + a], kbb = T[b * ld + b], kab = T[a * ld + b];
-          const double laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
-          const double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
-          double ck, sk, cl, sl;
+          const R kaa = T[a * ld + a], kbb = T[b * ld + b], kab = T[a * ld + b];
+          const R laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
+          const R xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+          R ck, sk, cl, sl;
           const bool bigk = rotation_of(kaa, kbb, kab, ck, sk);
           (void)rotation_of(laa, lbb, lab, cl, sl);
           if (k == l && bigk) *big = 1;
-          const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-          const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+          const R yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+          const R ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
           const int pa = systolic_next(a, np), pb = systolic_next(b, np);
           const int pc = systolic_next(cc, np), pd = systolic_next(d, np);
           Tn[pa * ld + pc] = cl * yac - sl * yad; Tn[pa * ld + pd] = sl * yac + cl * yad;
@@ -567,17 +596,17 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
           const int q = idx - nb2;
           const int x = q / np, l = q - x * np;
           const int cc = l, d = np + l;
-          const double laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
-          const double va = J[x * ld + cc], vb = J[x * ld + d];
-          double cl, sl;
+          const R laa = T[cc * ld + cc], lbb = T[d * ld + d], lab = T[cc * ld + d];
+          const R va = J[x * ld + cc], vb = J[x * ld + d];
+          R cl, sl;
           (void)rotation_of(laa, lbb, lab, cl, sl);
           Jn[x * ld + systolic_next(cc, np)] = cl * va - sl * vb;
           Jn[x * ld + systolic_next(d, np)] = sl * va + cl * vb;
         }
       }
       c.sync();
-      { double* t = T; T = Tn; Tn = t; }
-      { double* t = J; J = Jn; Jn = t; }
+      { R* t = T; T = Tn; Tn = t; }
+      { R* t = J; J = Jn; Jn = t; }
     }
     again = *big;
     c.sync();
@@ -593,16 +622,16 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, double** Tio, double** Talti
 // them) and (row, pair) items of J (kMJ).  Per item: the offset of its first element, the offsets
 // its results are stored at, and the pairs whose rotations it needs; offsets are below 2^16
 // (matrices of at most 64 x 65 doubles) and are kept two to a register.
-template <int LD, int kMT, int kMJ>
-FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio,
+template <int LD, int kMT, int kMJ, typename R>
+FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** Jaltio,
                        int dim, int jrows, int max_sweeps, int* big_out) {
   constexpr int ld = LD;
   const int pp = (dim + 1) & ~1;
   const int np = pp >> 1;
-  double* T = *Tio;
-  double* Tn = *Taltio;
-  double* J = *Jio;
-  double* Jn = *Jaltio;
+  R* T = *Tio;
+  R* Tn = *Taltio;
+  R* J = *Jio;
+  R* Jn = *Jaltio;
   unsigned tdesc0[kMT], tdesc1[kMT], tdesc2[kMT], jdesc0[kMJ], jdesc1[kMJ];
   bool tv[kMT], jv[kMJ];
 #pragma unroll
@@ -634,7 +663,7 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
       // every warp works out all np <= 32 rotations itself, lane q the one of pair q; the items then
       // fetch the two (one) they need with shuffles: no second barrier, no waiting for one warp
       const int lane = c.tid & 31;
-      double x0[kMT], x1[kMT], x2[kMT], x3[kMT], v0[kMJ], v1[kMJ];
+      R x0[kMT], x1[kMT], x2[kMT], x3[kMT], v0[kMJ], v1[kMJ];
 #pragma unroll
       for (int u = 0; u < kMT; ++u) {
         if (tv[u]) {
@@ -646,7 +675,7 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
       for (int u = 0; u < kMJ; ++u) {
         if (jv[u]) { const int jb = jdesc0[u] & 0xffffu; v0[u] = J[jb]; v1[u] = J[jb + np]; }
       }
-      double cq = 1.0, sq = 0.0;
+      R cq = 1.0, sq = 0.0;
       if (lane < np) {
         const int o = lane * (ld + 1);
         if (rotation_of(T[o], T[o + np * (ld + 1)], T[o + np], cq, sq) && c.tid < np) *big = 1;
@@ -654,11 +683,11 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
 #pragma unroll
       for (int u = 0; u < kMT; ++u) {
         const int tk = (tdesc0[u] >> 16) & 0xffu, tl = tdesc0[u] >> 24;
-        const double ck = __shfl_sync(0xffffffffu, cq, tk), sk = __shfl_sync(0xffffffffu, sq, tk);
-        const double cl = __shfl_sync(0xffffffffu, cq, tl), sl = __shfl_sync(0xffffffffu, sq, tl);
+        const R ck = __shfl_sync(0xffffffffu, cq, tk), sk = __shfl_sync(0xffffffffu, sq, tk);
+        const R cl = __shfl_sync(0xffffffffu, cq, tl), sl = __shfl_sync(0xffffffffu, sq, tl);
         if (tv[u]) {
-          const double yac = ck * x0[u] - sk * x2[u], yad = ck * x1[u] - sk * x3[u];
-          const double ybc = sk * x0[u] + ck * x2[u], ybd = sk * x1[u] + ck * x3[u];
+          const R yac = ck * x0[u] - sk * x2[u], yad = ck * x1[u] - sk * x3[u];
+          const R ybc = sk * x0[u] + ck * x2[u], ybd = sk * x1[u] + ck * x3[u];
           Tn[tdesc1[u] & 0xffffu] = cl * yac - sl * yad; Tn[tdesc1[u] >> 16] = sl * yac + cl * yad;
           Tn[tdesc2[u] & 0xffffu] = cl * ybc - sl * ybd; Tn[tdesc2[u] >> 16] = sl * ybc + cl * ybd;
         }
@@ -666,22 +695,22 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
 #pragma unroll
       for (int u = 0; u < kMJ; ++u) {
         const int jl = jdesc0[u] >> 16;
-        const double cl = __shfl_sync(0xffffffffu, cq, jl), sl = __shfl_sync(0xffffffffu, sq, jl);
+        const R cl = __shfl_sync(0xffffffffu, cq, jl), sl = __shfl_sync(0xffffffffu, sq, jl);
         if (jv[u]) {
           Jn[jdesc1[u] & 0xffffu] = cl * v0[u] - sl * v1[u];
           Jn[jdesc1[u] >> 16] = sl * v0[u] + cl * v1[u];
         }
       }
-      if (lane < np) { s.rc[lane] = cq; s.rs[lane] = sq; }     // same values from every warp: for the loops below
+      if (lane < np) { s.rc[lane] = (double)cq; s.rs[lane] = (double)sq; }     // same values from every warp: for the loops below
       // items beyond the per-thread lists (a smaller block than expected): offsets on the fly
       if (kMT * c.nt < np * np || kMJ * c.nt < jrows * np) c.sync();
       for (int idx = c.tid + kMT * c.nt; idx < np * np; idx += c.nt) {
         const int k = idx / np, l = idx - k * np;
         const int a = k, b = np + k, cc = l, d = np + l;
-        const double ck = s.rc[k], sk = s.rs[k], cl = s.rc[l], sl = s.rs[l];
-        const double xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
-        const double yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
-        const double ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
+        const R ck = (R)s.rc[k], sk = (R)s.rs[k], cl = (R)s.rc[l], sl = (R)s.rs[l];
+        const R xac = T[a * ld + cc], xad = T[a * ld + d], xbc = T[b * ld + cc], xbd = T[b * ld + d];
+        const R yac = ck * xac - sk * xbc, yad = ck * xad - sk * xbd;
+        const R ybc = sk * xac + ck * xbc, ybd = sk * xad + ck * xbd;
         const int pa = systolic_next(a, np), pb = systolic_next(b, np);
         const int pc = systolic_next(cc, np), pd = systolic_next(d, np);
         Tn[pa * ld + pc] = cl * yac - sl * yad; Tn[pa * ld + pd] = sl * yac + cl * yad;
@@ -690,14 +719,14 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
       for (int idx = c.tid + kMJ * c.nt; idx < jrows * np; idx += c.nt) {
         const int x = idx / np, l = idx - x * np;
         const int cc = l, d = np + l;
-        const double cl = s.rc[l], sl = s.rs[l];
-        const double va = J[x * ld + cc], vb = J[x * ld + d];
+        const R cl = (R)s.rc[l], sl = (R)s.rs[l];
+        const R va = J[x * ld + cc], vb = J[x * ld + d];
         Jn[x * ld + systolic_next(cc, np)] = cl * va - sl * vb;
         Jn[x * ld + systolic_next(d, np)] = sl * va + cl * vb;
       }
       c.sync();
-      { double* t = T; T = Tn; Tn = t; }
-      { double* t = J; J = Jn; Jn = t; }
+      { R* t = T; T = Tn; Tn = t; }
+      { R* t = J; J = Jn; Jn = t; }
     }
     again = *big;
     c.sync();
@@ -709,8 +738,8 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, double** Tio, double** Talti
 }
 #endif
 
-template <int LD>
-FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, double** Jio, double** Jaltio, int dim,
+template <int LD, typename R>
+FA_FN int jacobi(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** Jaltio, int dim,
                  int jrows, int max_sweeps, int* big_out) {
   *big_out = 0;
   if (dim < 2) return 0;
@@ -720,11 +749,11 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
   const int np = (dim + 1) >> 1;
   if (LD > 20 && np > 8) {
     if (np * np <= c.nt && jrows * np <= c.nt)
-      return jacobi_large<LD, 1, 1>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
-    return jacobi_large<LD, 2, 4>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+      return jacobi_large<LD, 1, 1, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+    return jacobi_large<LD, 2, 4, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
   }
 #endif
-  return jacobi_small<LD>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+  return jacobi_small<LD, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
 }
 
 // Refinement of approximate eigenvectors by matrix products (the iterative refinement for the
@@ -737,37 +766,41 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, double** Tio, double** Taltio, dou
 // rounds for a Jacobi sweep.  It only converges from close by: |E_ij| must be well below one, which
 // near-equal eigenvalues with a sizeable coupling entry violate -- those stay with the Jacobi sweeps.
 //
-// Starts from X = I, i.e. in the basis T is given in; the first step then needs no products
-// (S = T, Rm = 0).  Returns 1 with X in s.J and the eigenvalue estimates on the diagonal of T when
-// the corrections went below kRefineStop; 0 (T untouched) when the first corrections are above
+// Starts from X = I, i.e. in the basis T is given in -- the first step then needs no products
+// (S = T, Rm = 0) -- or, with from_x, from the matrix in s.J (the eigenvectors the fp32 sweeps found).
+// Returns 1 with X in s.J and the eigenvalue estimates on the diagonal of T when the corrections
+// went below kRefineStop; 0 (T untouched but for nothing) when the first corrections are above
 // kRefineTheta, the steps stop contracting or kMaxRefine steps are not enough.  Uses s.J, s.tmp and
 // s.M as scratch (pointers may come back swapped).
 template <int LD>
-FA_FN int refine_eig(const Ctx& c, Smem& s, int r) {
+FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
   constexpr int ld = LD;
   const double* T = s.T;
   double* X = s.J;       // current eigenvector estimate
   double* E = s.tmp;     // T X, then the correction E
   double* SR = s.M;      // S on and above the diagonal, Rm below it; becomes the next X
   const int ntri = r * (r + 1) / 2;
-  // ---- first step from X = I
-  double part = 0.0;
-  for (int idx = c.tid; idx < r * r; idx += c.nt) {
-    const int i = fast_div(idx, s.div_r), j = idx - i * r;
-    double e = 0.0;
-    if (i != j) {
-      const double tij = T[i * ld + j], tii = T[i * ld + i], tjj = T[j * ld + j];
-      if (tij * tij > (kJacobiTol * kJacobiTol) * fabs(tii * tjj) && tij * tij > 1e-280) {
-        e = tij * FA_RCP(tjj - tii);                 // equal diagonal entries: Inf, refused below
-        part = fmax(part, fabs(e) <= 1.7e308 ? fabs(e) : 1.7e308);
+  double part = 0.0, emax = 2.0 * kRefineTheta;      // from_x: the first full step must come out below kRefineTheta
+  int steps = 0;
+  if (!from_x) {
+    // ---- first step from X = I
+    for (int idx = c.tid; idx < r * r; idx += c.nt) {
+      const int i = fast_div(idx, s.div_r), j = idx - i * r;
+      double e = 0.0;
+      if (i != j) {
+        const double tij = T[i * ld + j], tii = T[i * ld + i], tjj = T[j * ld + j];
+        if (tij * tij > (kJacobiTol * kJacobiTol) * fabs(tii * tjj) && tij * tij > 1e-280) {
+          e = tij * FA_RCP(tjj - tii);                 // equal diagonal entries: Inf, refused below
+          part = fmax(part, fabs(e) <= 1.7e308 ? fabs(e) : 1.7e308);
+        }
       }
+      X[i * ld + j] = (i == j) ? 1.0 : e;
     }
-    X[i * ld + j] = (i == j) ? 1.0 : e;
+    emax = block_max(c, s, part);                      // its barrier also publishes X
+    if (!(emax <= kRefineTheta)) return 0;
+    for (int k = c.tid; k < r; k += c.nt) s.lam[k] = T[k * ld + k];
+    steps = 1;
   }
-  double emax = block_max(c, s, part);               // its barrier also publishes X
-  if (!(emax <= kRefineTheta)) return 0;
-  for (int k = c.tid; k < r; k += c.nt) s.lam[k] = T[k * ld + k];
-  int steps = 1;
   while (emax >= kRefineStop) {
     if (steps > kMaxRefine) return 0;
     const double prev = emax;
@@ -818,6 +851,56 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r) {
   s.count_refinements += steps;
   c.sync();
   return 1;
+}
+
+// Jacobi sweeps in fp32 on a copy of T (scaled to order one), for a round whose T is too far from
+// diagonal form for the refinement: sweeps until every |T_ij| is below half of kRefineTheta times
+// |T_jj - T_ii| in the swept copy (or the sweeps have converged as far as fp32 goes), then the
+// accumulated rotations are widened into s.J as the refinement's starting point.  A rotation round
+// costs about a third of the fp64 one when the block is latency-bound (up to 16 indices) and about
+// half when it is bound by shared-memory traffic (64 indices); what fp32 loses -- eigenvectors good
+// to 1e-6, orthogonal to 1e-6 -- the refinement restores in two of its steps.  s.T is only read.
+// The fp32 matrices live in s.tmp (T and its alternate) and s.M (J and its alternate).
+template <int LD>
+FA_FN void sweeps_fp32(const Ctx& c, Smem& s, int r) {
+  constexpr int ld = LD;
+  const int ppr = (r + 1) & ~1;
+  float* Tf = reinterpret_cast<float*>(s.tmp);
+  float* Ta = Tf + (LD - kLdPad) * LD;
+  float* Jf = reinterpret_cast<float*>(s.M);
+  float* Ja = Jf + (LD - kLdPad) * LD;
+  double part = 0.0;
+  for (int k = c.tid; k < r; k += c.nt) part = fmax(part, fmin(fabs(s.T[k * ld + k]), 1.7e308));
+  const double dmax = block_max(c, s, part);
+  const double scale = dmax > 0.0 ? 1.0 / dmax : 1.0;
+  for (int idx = c.tid; idx < ppr * ld; idx += c.nt) {
+    const int a = idx / ld, b = idx - a * ld;          // ld is a compile-time constant
+    Tf[idx] = (a < r && b < r) ? (float)(s.T[idx] * scale) : 0.0f;
+    Jf[idx] = (a == b) ? 1.0f : 0.0f;
+  }
+  c.sync();
+  for (int sweep = 0; sweep < kMaxSweepsF32; ++sweep) {
+    int big = 0;
+    s.count_sweeps_f32 += jacobi<LD, float>(c, s, &Tf, &Ta, &Jf, &Ja, r, r, 1, &big);
+    if (!big) break;
+    part = 0.0;
+    for (int idx = c.tid; idx < r * r; idx += c.nt) {
+      const int i = fast_div(idx, s.div_r), j = idx - i * r;
+      if (i != j) {
+        const float tij = Tf[i * ld + j], tii = Tf[i * ld + i], tjj = Tf[j * ld + j];
+        if (tij * tij > 1e-14f * fabsf(tii * tjj) && tij * tij > 1e-30f) {
+          const float th = fabsf(tij) / fabsf(tjj - tii);              // Inf for equal diagonal entries
+          part = fmax(part, th <= 3.0e38f ? (double)th : 1.7e308);
+        }
+      }
+    }
+    if (block_max(c, s, part) <= 0.5 * kRefineTheta) break;
+  }
+  for (int idx = c.tid; idx < r * r; idx += c.nt) {
+    const int i = fast_div(idx, s.div_r), j = idx - i * r;
+    s.J[i * ld + j] = (double)Jf[i * ld + j];
+  }
+  c.sync();
 }
 
 // ev[k] = T[k][k]; ord[q] = index of the q-th largest (ties by index).  All threads return
@@ -1348,8 +1431,17 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     // previous round's eigenbasis), the closer the further the rounds have converged: the refinement
     // is tried first, and each time it declines one Jacobi sweep is made, the coordinates are taken
     // to the swept basis and T is looked at again.
+    bool f32_tried = false;
     for (;;) {
       if (refine_eig<LD>(c, s, r)) break;
+      // far from diagonal: fp32 sweeps, then the refinement from what they found.  Only where a rotation
+      // round is bound by shared-memory traffic (more than 32 gradients: a quarter faster in fp32); with
+      // fewer the round costs the same in either precision and the extra refinement steps are a loss.
+      if (LD > 36 && !f32_tried) {
+        f32_tried = true;
+        sweeps_fp32<LD>(c, s, r);
+        if (refine_eig<LD>(c, s, r, true)) break;
+      }
       const int ppr = (r + 1) & ~1;                       // the sweeps work on an even number of indices
       for (int idx = c.tid; idx < ppr * ld; idx += c.nt) s.J[idx] = 0.0;
       if (ppr > r) for (int b = c.tid; b < ppr; b += c.nt) { s.T[r * ld + b] = 0.0; s.T[b * ld + r] = 0.0; }
@@ -1357,7 +1449,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       for (int a = c.tid; a < ppr; a += c.nt) s.J[a * (ld + 1)] = 1.0;
       c.sync();
       int big = 0;
-      sw += jacobi<LD>(c, s, &s.T, &s.tmp, &s.J, &s.M, r, r, 1, &big);   // M is free until the next weights
+      sw += jacobi<LD, double>(c, s, &s.T, &s.tmp, &s.J, &s.M, r, r, 1, &big);   // M is free until the next weights
       const bool last = !big || sw >= kMaxSweeps;
       if (big && last) status |= ST_EIG_SWEEPS;
       if (last) break;           // diagonal to rounding level (or given up): J holds the eigenvectors

@@ -10,7 +10,7 @@
 extern "C" int irls_host(const double* K, int p, int m, double lambda, double a, int iters, int start,
                          const double* A0, double tol, double* A, float* c, double* w, double* obj, double* S,
                          int* rounds, int workers, const unsigned char* counts, double cb, double ca,
-                         int* sweeps_out, int* refinements_out) {
+                         int* sweeps_out, int* refinements_out, int* sweeps_f32_out) {
   const size_t bytes = fa_irls::smem_bytes(p, 1);
   void* mem = calloc(bytes, 1);
   fa_irls::Ctx ctx{0, 1};
@@ -23,6 +23,7 @@ extern "C" int irls_host(const double* K, int p, int m, double lambda, double a,
   else st = fa_irls::run<68>(ctx, s, K, p, m, lambda, a, iters, start, A0, tol, o, workers, counts, cb, ca);
   if (sweeps_out) *sweeps_out = s.count_sweeps;
   if (refinements_out) *refinements_out = s.count_refinements;
+  if (sweeps_f32_out) *sweeps_f32_out = s.count_sweeps_f32;
   free(mem);
   return st;
 }

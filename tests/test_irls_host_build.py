@@ -35,7 +35,7 @@ def host(tmp_path_factory):
     assert r.returncode == 0, r.stderr
     lib = ctypes.CDLL(out)
     vp, i, d = ctypes.c_void_p, ctypes.c_int, ctypes.c_double
-    lib.irls_host.argtypes = [vp, i, i, d, d, i, i, vp, d, vp, vp, vp, vp, vp, vp, i, vp, d, d, vp, vp]
+    lib.irls_host.argtypes = [vp, i, i, d, d, i, i, vp, d, vp, vp, vp, vp, vp, vp, i, vp, d, d, vp, vp, vp]
     lib.irls_host.restype = i
     return lib
 
@@ -49,7 +49,7 @@ def run_host(lib, K, m, lam, iters, a=2.0, A0=None, tol=-1.0, counts=None, cb=1.
     w = np.zeros(nw)
     obj = np.zeros(iters)
     rounds = np.zeros(1, dtype=np.int32)
-    work = np.zeros(2, dtype=np.int32)
+    work = np.zeros(3, dtype=np.int32)
     cnt = np.zeros(64, dtype=np.uint8)
     if counts is not None:
         cnt[:nw] = counts
@@ -57,9 +57,9 @@ def run_host(lib, K, m, lam, iters, a=2.0, A0=None, tol=-1.0, counts=None, cb=1.
     st = lib.irls_host(K.ctypes.data, p, m, float(lam), float(a), iters, 0 if A0 is None else 2,
                        None if A0c is None else A0c.ctypes.data, float(tol), A.ctypes.data, c.ctypes.data,
                        w.ctypes.data, obj.ctypes.data, None, rounds.ctypes.data, 0 if counts is None else nw,
-                       cnt.ctypes.data, cb, ca, work.ctypes.data, work.ctypes.data + 4)
+                       cnt.ctypes.data, cb, ca, work.ctypes.data, work.ctypes.data + 4, work.ctypes.data + 8)
     return dict(status=st, A=A, c=c, w=w, objective=obj, rounds=int(rounds[0]), sweeps=int(work[0]),
-                refinements=int(work[1]))
+                refinements=int(work[1]), sweeps_f32=int(work[2]))
 
 
 @pytest.mark.parametrize("p,n,kind,m,lam,iters", IRLS_CASES)
@@ -95,8 +95,10 @@ def test_host_build_on_the_workload_recipes_and_the_work_it_takes(host, name, n)
     assert np.allclose(got["objective"], ref["objective"], rtol=0, atol=1e-9)
     assert fo.principal_angles(ref["Y"], G.T @ got["A"][:, :k]).max() < 1e-7
     assert fo.rel_l2(got["c"].astype(np.float64) @ G, ref["d"]) < 1e-6
-    print(f"{w.name}: {got['sweeps']} Jacobi sweeps, {got['refinements']} refinement steps in {w.iters} rounds")
-    assert got["sweeps"] <= 3 * w.iters and got["refinements"] >= w.iters
+    print(f"{w.name}: {got['sweeps_f32']} fp32 and {got['sweeps']} fp64 Jacobi sweeps, {got['refinements']} refinement "
+          f"steps in {w.iters} rounds")
+    assert got["sweeps"] + got["sweeps_f32"] <= 3 * w.iters and got["refinements"] >= w.iters
+    assert (got["sweeps_f32"] > 0) == (w.p > 32)         # fp32 sweeps only where the rounds are bound by shared-memory traffic
 
 
 def test_host_build_with_workers_that_hold_several_gradients(host):
