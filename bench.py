@@ -204,6 +204,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--min-time", type=float, default=1.0, help="length of the timed region in seconds, at least")
+    ap.add_argument("--kernel-reps", type=int, default=100, help="launches per kernel for the per-kernel medians "
+                    "(fewer under a profiler)")
     ap.add_argument("--replicas", action="store_true",
                     help="N > 1: N independent copies of the single-GPU step (weak scaling) instead of the n-sharded step")
     ap.add_argument("--worker-resident", action="store_true",
@@ -329,7 +331,7 @@ def main():
     kernels, roofline, step_hbm = None, None, None
     peak, peak_src = measured_peaks()
     if mode != "worker-resident":
-        reps = 100 if w.p * w.n * w.itemsize < 4e9 else 30
+        reps = max(3, args.kernel_reps if w.p * w.n * w.itemsize < 4e9 else min(args.kernel_reps, 30))
         K = torch.empty((w.p, w.p), dtype=torch.float64, device="cuda")
         cvec = torch.full((w.p,), 1.0 / w.p, dtype=torch.float32, device="cuda")
         wsk = fa.new_workspace(Gs[0], w.m)

@@ -234,6 +234,15 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   const bool issuer = role == 0 && lane == 0;
   if (issuer)
     for (int v = 0; v < kQuadDepth; ++v) issue(tfirst + v * tstride, v);
+  // the team's loads in flight when it gives up at tile t (stage s0, phase ph0) -- this stage's and the
+  // following ones' -- must land before the block can exit: these waits keep the long limit
+  auto drain = [&](int t, int s0, uint32_t ph0) {
+    if (!issuer) return;
+    for (int k = 0; k < kQuadDepth; ++k) {
+      if (t + k * tstride < ntiles) (void)mbar_wait(&mybars[s0], ph0);
+      if (++s0 == kQuadDepth) { s0 = 0; ph0 ^= 1u; }
+    }
+  };
 
   float acc[kQuadAcc];
   double dacc[kQuadAcc / 32];
@@ -247,62 +256,58 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
   uint32_t phase = 0;
   for (int t = tfirst; t < ntiles; t += tstride) {
     // Giving up must be a decision of the whole team: its four warps meet at the team's barrier after
-    // every tile, so a warp whose wait ran out skips the tile, raises the team's flag and still goes
-    // to the barrier; behind it all four read the flag and leave together.
-    const bool ok = __any_sync(0xffffffffu, mbar_wait(&mybars[s], phase, prm.wait_cycles));
-    if (!ok && lane == 0) {
-      if (prm.status) atomicOr(prm.status, kStTimeout);
-      *reinterpret_cast<volatile int*>(&aborted[team]) = 1;
+    // every tile, so a warp whose wait ran out raises the team's flag and still goes to that barrier;
+    // behind it all four read the flag and leave together.  (The lanes of a warp poll on their own;
+    // once any of them has seen the phase complete, it is complete.)
+    if (!__any_sync(0xffffffffu, mbar_wait(&mybars[s], phase, prm.wait_cycles))) {
+      if (lane == 0) {
+        if (prm.status) atomicOr(prm.status, kStTimeout);
+        *reinterpret_cast<volatile int*>(&aborted[team]) = 1;
+      }
+      team_barrier(team);
+      drain(t, s, phase);
+      break;
     }
-    if (ok) {
-      const char* sbase = mystages + (size_t)s * kStageBytes;
-      if (role < 2) {
-  #pragma unroll 1
-        for (int cg = lane; cg < kTileCols / 2; cg += 32) {
-          const char* ptr = sbase + rowbase + cg * 8;
-          float x[16][2];
-  #pragma unroll
-          for (int i = 0; i < 16; ++i) SmemVec<float, 2>::load(ptr + i * kRowBytes, x[i]);
-          int idx = 0;
-  #pragma unroll
-          for (int i = 0; i < 16; ++i)
-  #pragma unroll
-            for (int j = i; j < 16; ++j) {
-              acc[idx] = fmaf(x[i][0], x[j][0], acc[idx]);
-              acc[idx] = fmaf(x[i][1], x[j][1], acc[idx]);
-              ++idx;
-            }
-        }
-      } else {
-  #pragma unroll 1
-        for (int cg = lane; cg < kTileCols / 2; cg += 32) {
-          const char* pa = sbase + rowbase + cg * 8;
-          const char* pb = sbase + 16 * kRowBytes + cg * 8;
-          float a[8][2], b[16][2];
-  #pragma unroll
-          for (int i = 0; i < 8; ++i) SmemVec<float, 2>::load(pa + i * kRowBytes, a[i]);
-  #pragma unroll
-          for (int j = 0; j < 16; ++j) SmemVec<float, 2>::load(pb + j * kRowBytes, b[j]);
-  #pragma unroll
-          for (int i = 0; i < 8; ++i)
-  #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
-              acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
-            }
-        }
+    const char* sbase = mystages + (size_t)s * kStageBytes;
+    if (role < 2) {
+#pragma unroll 1
+      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+        const char* ptr = sbase + rowbase + cg * 8;
+        float x[16][2];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) SmemVec<float, 2>::load(ptr + i * kRowBytes, x[i]);
+        int idx = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+#pragma unroll
+          for (int j = i; j < 16; ++j) {
+            acc[idx] = fmaf(x[i][0], x[j][0], acc[idx]);
+            acc[idx] = fmaf(x[i][1], x[j][1], acc[idx]);
+            ++idx;
+          }
+      }
+    } else {
+#pragma unroll 1
+      for (int cg = lane; cg < kTileCols / 2; cg += 32) {
+        const char* pa = sbase + rowbase + cg * 8;
+        const char* pb = sbase + 16 * kRowBytes + cg * 8;
+        float a[8][2], b[16][2];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) SmemVec<float, 2>::load(pa + i * kRowBytes, a[i]);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) SmemVec<float, 2>::load(pb + j * kRowBytes, b[j]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
+            acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
+          }
       }
     }
     team_barrier(team);                  // all four parts are done with the stage
-    if (*reinterpret_cast<volatile int*>(&aborted[team])) {
-      if (issuer) {   // the team's loads in flight (this stage's and the following ones') must land: long limit
-        int s2 = s;
-        uint32_t ph2 = phase;
-        for (int k = 0; k < kQuadDepth; ++k) {
-          if (t + k * tstride < ntiles) (void)mbar_wait(&mybars[s2], ph2);
-          if (++s2 == kQuadDepth) { s2 = 0; ph2 ^= 1u; }
-        }
-      }
+    if (*reinterpret_cast<volatile int*>(&aborted[team])) {      // another warp of the team gave up on this tile
+      drain(t, s, phase);
       break;
     }
     if (issuer) {
