@@ -63,8 +63,17 @@ constexpr double kRankRel = 1e-12;     // eigenvalue <= this * largest: directio
 constexpr double kJacobiTol = 1e-17;   // rotate when |a_pq| > tol * sqrt(|a_pp a_qq|)
 constexpr double kJacobiBig = 1e-6;    // sweep again while some rotated |a_pq| exceeded this (relative)
 constexpr int kMaxSweeps = 40;
-constexpr double kRefineTheta = 0.3;   // refinement is tried when every |T_ij| <= this * |T_jj - T_ii|
-constexpr double kRefineStop = 1e-8;   // ... and has converged when a step's largest correction is below this
+// The refinement is tried when every |T_ij| <= theta * |T_jj - T_ii|, has converged when a step's largest
+// correction is below kRefineStop, and is given up when a step's largest correction is not below
+// `contract` times the one before.  Up to 32 gradients a declined attempt is cheap next to a sweep, so the
+// reach is set wide (measured on the workloads' spectra: 13 sweeps + 51 steps instead of 16 + 45 at p = 15,
+// 20 + 90 instead of 26 + 82 at p = 31); above, a failed attempt costs a quarter of a sweep and the tighter
+// pair is faster (p = 63 at its full size: 2.9 ms per call against 3.8 ms).
+template <int LD> struct RefineLimits {
+  static constexpr double theta = LD > 36 ? 0.3 : 0.5;
+  static constexpr double contract = LD > 36 ? 0.5 : 0.7;
+};
+constexpr double kRefineStop = 1e-8;
 constexpr int kMaxRefine = 8;          // steps after which a refinement that has not converged is given up
 constexpr int kMaxSweepsF32 = 12;      // fp32 sweeps per round before the fp64 sweeps take over
 constexpr int kMaxP = 64;
@@ -770,7 +779,7 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** 
 // (S = T, Rm = 0) -- or, with from_x, from the matrix in s.J (the eigenvectors the fp32 sweeps found).
 // Returns 1 with X in s.J and the eigenvalue estimates on the diagonal of T when the corrections
 // went below kRefineStop; 0 (T untouched but for nothing) when the first corrections are above
-// kRefineTheta, the steps stop contracting or kMaxRefine steps are not enough.  Uses s.J, s.tmp and
+// the reach (RefineLimits), the steps stop contracting or kMaxRefine steps are not enough.  Uses s.J, s.tmp and
 // s.M as scratch (pointers may come back swapped).
 template <int LD>
 FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
@@ -780,7 +789,8 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
   double* E = s.tmp;     // T X, then the correction E
   double* SR = s.M;      // S on and above the diagonal, Rm below it; becomes the next X
   const int ntri = r * (r + 1) / 2;
-  double part = 0.0, emax = 2.0 * kRefineTheta;      // from_x: the first full step must come out below kRefineTheta
+  constexpr double kRefineTheta = RefineLimits<LD>::theta, kRefineContract = RefineLimits<LD>::contract;
+  double part = 0.0, emax = kRefineTheta / kRefineContract;   // from_x: the first full step must come out below kRefineTheta
   int steps = 0;
   if (!from_x) {
     // ---- first step from X = I
@@ -838,7 +848,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
       E[i * ld + j] = e;
     }
     emax = block_max(c, s, part);                    // its barrier: every thread is done with SR, E is published
-    if (!(emax <= 0.5 * prev) && emax > 1e-12) return 0;
+    if (!(emax <= kRefineContract * prev) && emax > 1e-12) return 0;
     // ---- X <- X + X E  (into SR's buffer, which then changes roles with X's)
     matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, X, E, [&](int i, int j, double v) { SR[i * ld + j] = X[i * ld + j] + v; });
     c.sync();
@@ -854,7 +864,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
 }
 
 // Jacobi sweeps in fp32 on a copy of T (scaled to order one), for a round whose T is too far from
-// diagonal form for the refinement: sweeps until every |T_ij| is below half of kRefineTheta times
+// diagonal form for the refinement: sweeps until every |T_ij| is below half of the refinement's reach times
 // |T_jj - T_ii| in the swept copy (or the sweeps have converged as far as fp32 goes), then the
 // accumulated rotations are widened into s.J as the refinement's starting point.  A rotation round
 // costs about a third of the fp64 one when the block is latency-bound (up to 16 indices) and about
@@ -894,7 +904,7 @@ FA_FN void sweeps_fp32(const Ctx& c, Smem& s, int r) {
         }
       }
     }
-    if (block_max(c, s, part) <= 0.5 * kRefineTheta) break;
+    if (block_max(c, s, part) <= 0.5 * RefineLimits<LD>::theta) break;
   }
   for (int idx = c.tid; idx < r * r; idx += c.nt) {
     const int i = fast_div(idx, s.div_r), j = idx - i * r;
@@ -956,7 +966,8 @@ FA_FN void term_of(double u, double a, double& contrib, double& denom) {
 // beta = 1/2, i.e. cb = 1, ca = 0.  With ca > 0 a weight can be negative.
 template <int LD>
 FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int k0, int r, int p,
-                                   double coef, bool uniform, double a, double cb = 1.0, double ca = 0.0) {
+                                   double coef, bool uniform, double a, double cb = 1.0, double ca = 0.0,
+                                   bool want_objective = true) {
   constexpr int ld = LD;
   double part = 0.0;
   for (int i = c.tid; i < p; i += c.nt) {
@@ -1040,8 +1051,11 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
       s.M[i * ld + i] = s.w[i] + acc;
     }
   }
-  double obj = block_sum(c, s, part);   // contains the barriers that publish M and w
-  return obj;
+  if (!want_objective) {                 // nobody asked for the value of Eq. (5): the sum over the block is skipped
+    c.sync();                            // publishes M and w
+    return 0.0;
+  }
+  return block_sum(c, s, part);          // its barrier also publishes M and w
 }
 
 // The same for workers that hold several gradients each (rows of one worker are consecutive):
@@ -1472,8 +1486,9 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     { double* x = s.Aacc; s.Aacc = s.M; s.M = x; }
 
     // ---- terms of Eq. (5) at the new subspace, and the next round's weights
+    const bool want_obj = o.obj != nullptr || tol >= 0.0;
     double obj = grouped ? weights_and_objective_grouped<LD>(c, s, s.P, m_eff, r, p, coef, false, a)
-                         : weights_and_objective<LD>(c, s, s.P, m_eff, r, p, coef, false, a, cb, ca);
+                         : weights_and_objective<LD>(c, s, s.P, m_eff, r, p, coef, false, a, cb, ca, want_obj);
     if (o.obj && c.tid == 0) o.obj[t] = obj;
     if (tol >= 0.0 && t >= 1 && fabs(prev_obj - obj) <= tol) {      // same value in every thread
       rounds = t + 1;
