@@ -331,20 +331,6 @@ def main():
     kernels, roofline, step_hbm = None, None, None
     peak, peak_src = measured_peaks()
 
-    # Context for the fractions: the peak in MEASURED_PEAKS.json is a COPY (reads + writes), and a pass that
-    # mostly reads can exceed it.  A read-only probe (torch.sum over 2 GiB of fp32, best of 5) shows how far.
-    def read_only_probe():
-        x = torch.empty(1 << 29, dtype=torch.float32, device="cuda").fill_(1.0)
-        best = None
-        for _ in range(6):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); x.sum(); b.record(stream)
-            torch.cuda.synchronize()
-            t = a.elapsed_time(b)
-            best = t if best is None or t < best else best
-        del x
-        return (4 << 29) / (best * 1e-3) / 1e9
-    read_peak = read_only_probe() if (rank == 0 and mode == "single") else None
     if mode != "worker-resident":
         reps = max(3, args.kernel_reps if w.p * w.n * w.itemsize < 4e9 else min(args.kernel_reps, 30))
         K = torch.empty((w.p, w.p), dtype=torch.float64, device="cuda")
@@ -374,8 +360,6 @@ def main():
                               "(dram__bytes_read 240.07 MB, dram__bytes_write 10.7 MB); reads scaled by n, writes not")
         roofline = {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
                     "unit": "GB/s", "frac": gram_gbs / peak, "frac_of_nominal_8TBs": gram_gbs / 8000.0,
-                    "frac_of_read_only_probe": (gram_gbs / read_peak) if read_peak else None,
-                    "read_only_probe_gbs": read_peak,
                     "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_src,
                     "bytes_per_launch": int(gram_bytes), "ms_per_launch": t_gram}
         kernels = {"gram_ms": t_gram, "irls_ms": t_irls, "combine_ms": t_comb, "launches_timed": reps,

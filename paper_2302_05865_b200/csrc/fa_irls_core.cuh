@@ -117,6 +117,7 @@ FA_HD int leading_dim(int p) { return (p <= 16 ? 16 : (p <= 32 ? 32 : 64)) + kLd
 // Shared-memory image.  Matrices are (ld - kLdPad) x ld doubles.
 struct Smem {
   double *T, *J, *P, *M, *Aacc, *tmp;   // six matrix buffers, rotated by pointer swaps
+  double *V0, *V1;                       // up to 32 gradients: two more, for T X of the refinement (null above)
   double *kd, *dinv, *fn, *u, *w, *wused, *ev, *red;
   double *lam, *rdiag;                   // refinement: eigenvalue estimates, diagonal of I - X^T X
   double *rc, *rs;                       // rotation cos / sin per pair
@@ -138,7 +139,7 @@ struct Smem {
 FA_HD size_t smem_bytes(int p, int nt) {
   int ld = leading_dim(p);
   int pp = ld - kLdPad;
-  size_t doubles = (size_t)6 * pp * ld + (size_t)14 * pp + (nt < 128 ? 128 : nt) + 2 * (pp / 2 + 1);
+  size_t doubles = (size_t)(ld <= 36 ? 8 : 6) * pp * ld + (size_t)14 * pp + (nt < 128 ? 128 : nt) + 2 * (pp / 2 + 1);
   size_t ints = (size_t)2 * (pp / 2 + 1) + 4 * pp + 8 + (size_t)(pp * (pp - 1) / 2 + 1) / 2;
   return doubles * sizeof(double) + ints * sizeof(int) + 64;
 }
@@ -154,6 +155,8 @@ FA_FN void carve(Smem& s, void* base, int p, int nt) {
   s.M = d; d += (size_t)pp * ld;
   s.Aacc = d; d += (size_t)pp * ld;
   s.tmp = d; d += (size_t)pp * ld;
+  s.V0 = s.V1 = nullptr;
+  if (ld <= 36) { s.V0 = d; d += (size_t)pp * ld; s.V1 = d; d += (size_t)pp * ld; }
   s.kd = d; d += pp; s.dinv = d; d += pp; s.fn = d; d += pp; s.u = d; d += pp;
   s.w = d; d += pp; s.wused = d; d += pp; s.ev = d; d += pp;
   s.gtr = d; d += pp; s.gu = d; d += pp; s.gw = d; d += pp; s.gwused = d; d += pp; s.ginv = d; d += pp;
@@ -811,14 +814,26 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
     for (int k = c.tid; k < r; k += c.nt) s.lam[k] = T[k * ld + k];
     steps = 1;
   }
+  // V = T X.  Up to 32 gradients it has buffers of its own and is carried along (T (X + X E) = V + V E: the
+  // product by E that updates X updates V in the same phase, on other warps); above, there is no room
+  // and it is formed afresh in every step, in E's buffer.
+  double* V = s.V0;
+  double* Vn = s.V1;
+  const bool carry = V != nullptr;
+  if (carry && emax >= kRefineStop) {
+    matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, T, X, [&](int i, int j, double v) { V[i * ld + j] = v; });
+    c.sync();
+  }
   while (emax >= kRefineStop) {
     if (steps > kMaxRefine) return 0;
     const double prev = emax;
-    // ---- E <- T X
-    matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, T, X, [&](int i, int j, double v) { E[i * ld + j] = v; });
-    c.sync();
+    if (!carry) {
+      V = E;
+      matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, T, X, [&](int i, int j, double v) { V[i * ld + j] = v; });
+      c.sync();
+    }
     // ---- S = X^T (T X) on and above the diagonal, Rm = I - X^T X below it (its diagonal -> rdiag)
-    matmul<1, LD, LD, 1>(c, r, r, r, s.div_tr, X, E, [&](int i, int j, double v) { if (i <= j) SR[i * ld + j] = v; });
+    matmul<1, LD, LD, 1>(c, r, r, r, s.div_tr, X, V, [&](int i, int j, double v) { if (i <= j) SR[i * ld + j] = v; });
     matmul<1, LD, LD, 1>(c, r, r, r, s.div_tr, X, X,
                          [&](int i, int j, double v) { if (i == j) s.rdiag[i] = 1.0 - v; else if (i > j) SR[i * ld + j] = -v; },
                          ((r + 7) >> 3) * ((r + 7) >> 3));
@@ -849,9 +864,13 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
     }
     emax = block_max(c, s, part);                    // its barrier: every thread is done with SR, E is published
     if (!(emax <= kRefineContract * prev) && emax > 1e-12) return 0;
-    // ---- X <- X + X E  (into SR's buffer, which then changes roles with X's)
+    // ---- X <- X + X E  (into SR's buffer, which then changes roles with X's), and V <- V + V E
     matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, X, E, [&](int i, int j, double v) { SR[i * ld + j] = X[i * ld + j] + v; });
+    if (carry && emax >= kRefineStop)          // (the last step's V would not be used)
+      matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, V, E, [&](int i, int j, double v) { Vn[i * ld + j] = V[i * ld + j] + v; },
+                           ((r + 7) >> 3) * ((r + 7) >> 3));
     c.sync();
+    if (carry) { double* t = V; V = Vn; Vn = t; }
     { double* t = X; X = SR; SR = t; }
     ++steps;
   }
