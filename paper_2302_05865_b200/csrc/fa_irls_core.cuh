@@ -757,15 +757,29 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** 
   if (dim < 2) return 0;
 #ifndef FA_IRLS_HOST
   // item slots per thread are compile-time (slots without an item still cost their instructions):
-  // one of each up to 16 pairs with 512 threads, two blocks and four J items up to 32 pairs
+  // one of each up to 16 pairs with 512 threads, two blocks and three or four J items up to 32 pairs
   const int np = (dim + 1) >> 1;
-  if (LD > 20 && np > 8) {
-    if (np * np <= c.nt && jrows * np <= c.nt)
+  if constexpr (LD > 20) {
+    // Only the variants a kernel needs are compiled into it -- every further one costs it registers (the
+    // 512-thread kernels have 128 each: with all variants inlined the p = 31 call was 10 % slower).  So
+    // the kernels for more than 16 gradients run every size, a small rank included, through jacobi_large.
+    // Up to 32 gradients (512 threads) one item of each kind always suffices.  Above, the fp32 sweeps
+    // (the ones that normally run) come with three or four J items; the fp64 fallback with four.
+    if constexpr (LD <= 36) {
       return jacobi_large<LD, 1, 1, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
-    return jacobi_large<LD, 2, 4, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+    } else if constexpr (sizeof(R) == 4) {
+      if (np * np <= 2 * c.nt && jrows * np <= 3 * c.nt)    // e.g. 49 indices after 15 identical gradients of 63
+        return jacobi_large<LD, 2, 3, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+      return jacobi_large<LD, 2, 4, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+    } else {
+      return jacobi_large<LD, 2, 4, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+    }
+  } else {
+    return jacobi_small<LD, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
   }
-#endif
+#else
   return jacobi_small<LD, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+#endif
 }
 
 // Refinement of approximate eigenvectors by matrix products (the iterative refinement for the
@@ -819,7 +833,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
   // and it is formed afresh in every step, in E's buffer.
   double* V = s.V0;
   double* Vn = s.V1;
-  const bool carry = V != nullptr;
+  constexpr bool carry = LD <= 36;               // (= the kernels whose shared memory holds V0 and V1)
   if (carry && emax >= kRefineStop) {
     matmul<LD, 1, LD, 1>(c, r, r, r, s.div_tr, T, X, [&](int i, int j, double v) { V[i * ld + j] = v; });
     c.sync();
