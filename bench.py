@@ -349,15 +349,19 @@ def main():
         gram_gbs = gram_bytes / (t_gram * 1e-3) / 1e9
         comb_gbs = comb_bytes / (t_comb * 1e-3) / 1e9
         step_gbs = w_full.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
-        # DRAM bytes of one Gram launch: counters of one ncu capture of this kernel (fp32, p = 15, tensor-fed
-        # kernel, n = 4,000,000): 240.07 MB read for 240.00 MB of gradients, 10.7 MB written.  The reads grow with
-        # n (two row classes re-read 1.6 % when n * 4 is not a multiple of 16), the writes are per block and do not.
+        # DRAM bytes of one Gram launch, from ncu captures of the kernels as they stand, on cases small enough to
+        # capture: fp32 p = 15 at n = 4,000,002 (rows in two alignment classes, as in the full workload): 240.11 MB
+        # read for 240.00 MB of gradients, 10.9 MB written; fp32 p = 31 at n = 2,000,000: 248.10 MB read for
+        # 248.00 MB, 4.1 MB written.  The reads grow with n; the writes are per block and do not.
         traffic, traffic_source = None, None
         if w.p == 15 and w.dtype == "f32" and w.n >= 4096:
-            reread = 1.016 if (w.n * 4) % 16 else 1.0
-            traffic = int(240.07e6 * (w.n / 4_000_000) * reread + 10.7e6)
-            traffic_source = ("ncu capture of gramtm::gram_tri_tm_kernel<float,2,15> at n = 4,000,000 "
-                              "(dram__bytes_read 240.07 MB, dram__bytes_write 10.7 MB); reads scaled by n, writes not")
+            traffic = int(240.107e6 * (w.n / 4_000_002) + 10.9e6)
+            traffic_source = ("ncu capture of gramtm::gram_tri_tm_kernel<float,2,15> at n = 4,000,002 "
+                              "(dram__bytes_read 240.11 MB, dram__bytes_write 10.9 MB); reads scaled by n, writes not")
+        elif w.p == 31 and w.dtype == "f32" and w.n >= 4096:
+            traffic = int(248.10e6 * (w.n / 2_000_000) + 4.1e6)
+            traffic_source = ("ncu capture of gram_quad_tm_kernel at n = 2,000,000 "
+                              "(dram__bytes_read 248.10 MB, dram__bytes_write 4.1 MB); reads scaled by n, writes not")
         roofline = {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
                     "unit": "GB/s", "frac": gram_gbs / peak, "frac_of_nominal_8TBs": gram_gbs / 8000.0,
                     "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_src,
