@@ -130,7 +130,16 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
       float x[PB][V];
 #pragma unroll
       for (int i = 0; i < PB; ++i) {
-        SmemVec<T, V>::load(sbase + rowoff[i] + cg * (V * S), x[i]);
+        if constexpr (S == 4 && V == 2 && PB > 12) {
+          // two columns half a tile apart, one 4-byte load each: an 8-byte load of neighbours would put both
+          // factors of every product into the same register bank (every other FMA then takes a second
+          // dispatch cycle).  Up to 12 rows the pass is bound by the loads of the tiles and the fewer, wider
+          // shared loads are the better choice.
+          x[i][0] = *reinterpret_cast<const float*>(sbase + rowoff[i] + cg * 4);
+          x[i][1] = *reinterpret_cast<const float*>(sbase + rowoff[i] + (cg + groups) * 4);
+        } else {
+          SmemVec<T, V>::load(sbase + rowoff[i] + cg * (V * S), x[i]);
+        }
         if (i >= prm.p) {
 #pragma unroll
           for (int e = 0; e < V; ++e) x[i][e] = 0.f;
