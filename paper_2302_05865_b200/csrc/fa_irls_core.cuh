@@ -634,7 +634,7 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
 // them) and (row, pair) items of J (kMJ).  Per item: the offset of its first element, the offsets
 // its results are stored at, and the pairs whose rotations it needs; offsets are below 2^16
 // (matrices of at most 64 x 65 doubles) and are kept two to a register.
-template <int LD, int kMT, int kMJ, typename R>
+template <int LD, int kMT, int kMJ, typename R, bool kOnce = false>
 FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** Jaltio,
                        int dim, int jrows, int max_sweeps, int* big_out) {
   constexpr int ld = LD;
@@ -688,15 +688,28 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
         if (jv[u]) { const int jb = jdesc0[u] & 0xffffu; v0[u] = J[jb]; v1[u] = J[jb + np]; }
       }
       R cq = 1.0, sq = 0.0;
-      if (lane < np) {
+      if (kOnce) {
+        // the first warp alone works out the rotations and leaves them in shared memory: a second barrier,
+        // but the other warps' arithmetic pipes stay free of fifteen more copies of the same work
+        if (c.tid < np) {
+          const int o = c.tid * (ld + 1);
+          if (rotation_of(T[o], T[o + np * (ld + 1)], T[o + np], cq, sq)) *big = 1;
+          s.rc[c.tid] = (double)cq; s.rs[c.tid] = (double)sq;
+        }
+        c.sync();
+      } else if (lane < np) {
         const int o = lane * (ld + 1);
         if (rotation_of(T[o], T[o + np * (ld + 1)], T[o + np], cq, sq) && c.tid < np) *big = 1;
       }
 #pragma unroll
       for (int u = 0; u < kMT; ++u) {
         const int tk = (tdesc0[u] >> 16) & 0xffu, tl = tdesc0[u] >> 24;
-        const R ck = __shfl_sync(0xffffffffu, cq, tk), sk = __shfl_sync(0xffffffffu, sq, tk);
-        const R cl = __shfl_sync(0xffffffffu, cq, tl), sl = __shfl_sync(0xffffffffu, sq, tl);
+        R ck, sk, cl, sl;
+        if (kOnce) { ck = (R)s.rc[tk]; sk = (R)s.rs[tk]; cl = (R)s.rc[tl]; sl = (R)s.rs[tl]; }
+        else {
+          ck = __shfl_sync(0xffffffffu, cq, tk); sk = __shfl_sync(0xffffffffu, sq, tk);
+          cl = __shfl_sync(0xffffffffu, cq, tl); sl = __shfl_sync(0xffffffffu, sq, tl);
+        }
         if (tv[u]) {
           const R yac = ck * x0[u] - sk * x2[u], yad = ck * x1[u] - sk * x3[u];
           const R ybc = sk * x0[u] + ck * x2[u], ybd = sk * x1[u] + ck * x3[u];
@@ -707,15 +720,17 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
 #pragma unroll
       for (int u = 0; u < kMJ; ++u) {
         const int jl = jdesc0[u] >> 16;
-        const R cl = __shfl_sync(0xffffffffu, cq, jl), sl = __shfl_sync(0xffffffffu, sq, jl);
+        R cl, sl;
+        if (kOnce) { cl = (R)s.rc[jl]; sl = (R)s.rs[jl]; }
+        else { cl = __shfl_sync(0xffffffffu, cq, jl); sl = __shfl_sync(0xffffffffu, sq, jl); }
         if (jv[u]) {
           Jn[jdesc1[u] & 0xffffu] = cl * v0[u] - sl * v1[u];
           Jn[jdesc1[u] >> 16] = sl * v0[u] + cl * v1[u];
         }
       }
-      if (lane < np) { s.rc[lane] = (double)cq; s.rs[lane] = (double)sq; }     // same values from every warp: for the loops below
+      if (!kOnce && lane < np) { s.rc[lane] = (double)cq; s.rs[lane] = (double)sq; }     // same values from every warp: for the loops below
       // items beyond the per-thread lists (a smaller block than expected): offsets on the fly
-      if (kMT * c.nt < np * np || kMJ * c.nt < jrows * np) c.sync();
+      if (!kOnce && (kMT * c.nt < np * np || kMJ * c.nt < jrows * np)) c.sync();
       for (int idx = c.tid + kMT * c.nt; idx < np * np; idx += c.nt) {
         const int k = idx / np, l = idx - k * np;
         const int a = k, b = np + k, cc = l, d = np + l;
@@ -766,7 +781,7 @@ FA_FN int jacobi(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio, R** 
     // Up to 32 gradients (512 threads) one item of each kind always suffices.  Above, the fp32 sweeps
     // (the ones that normally run) come with three or four J items; the fp64 fallback with four.
     if constexpr (LD <= 36) {
-      return jacobi_large<LD, 1, 1, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
+      return jacobi_large<LD, 1, 1, R, true>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
     } else if constexpr (sizeof(R) == 4) {
       if (np * np <= 2 * c.nt && jrows * np <= 3 * c.nt)    // e.g. 49 indices after 15 identical gradients of 63
         return jacobi_large<LD, 2, 3, R>(c, s, Tio, Taltio, Jio, Jaltio, dim, jrows, max_sweeps, big_out);
