@@ -482,7 +482,10 @@ FA_FN int systolic_next(int x, int np) {
 //     column pair itself and gets the one of its row pair from another lane of its warp by a
 //     shuffle: one barrier per round and nothing else between threads;
 //   * more pairs (jacobi_large): several items per thread; every warp works out all rotations
-//     (lane q: pair q) and the items fetch theirs by shuffles -- still one barrier per round.
+//     (lane q: pair q) and the items fetch theirs by shuffles -- still one barrier per round; or
+//     (kOnce, used up to 16 pairs in fp64) the first warp alone works them out and a second barrier
+//     publishes them: sixteen warps repeating the fp64 divisions and square roots kept the fp64
+//     pipe busier than the extra barrier costs.
 // A full sweep (pp - 1 rounds) returns every index to its own position, and sweeps are never cut
 // short.  On return *Tio / *Jio point at the buffers that hold the results.  Returns the sweeps made.
 // Up to 8 pairs on the device; any size on the host.
