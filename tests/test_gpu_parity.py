@@ -51,6 +51,10 @@ LADDER = [
     # the output pass reads 16-byte vectors and hands half of them to the neighbouring thread
     (15, 65_538, "noisy_mean", False, 2), (16, 10, "gauss", False, 0), (3, 8, "gauss", False, 2),
     (9, 130, "noisy_mean", False, 0), (33, 4_098, "dup_zero", False, 2), (64, 1_026, "gauss", False, 0),
+    # fp32, 13 to 16 rows in the tensor-fed kernel, rows in one, two and four alignment classes (4-byte operand loads
+    # of columns half a tile apart; the tile step is 256 or 252 columns)
+    (13, 20_001, "noisy_mean", False, 0), (14, 30_002, "gauss", False, 0), (16, 50_003, "dup_zero", False, 0),
+    (16, 40_002, "noisy_mean", False, 2), (13, 8_192, "gauss", False, 4),
     # bf16, p > 16, 16-byte aligned rows: the tensor-core kernel
     (17, 64, "gauss", True, 0), (33, 264, "noisy_mean", True, 0), (63, 4_096, "dup_zero", True, 0),
     (64, 65_536, "gauss", True, 0), (31, 1_000_000, "dup_zero", True, 8), (48, 300_008, "noisy_mean", True, 0),
