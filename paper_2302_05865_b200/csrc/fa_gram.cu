@@ -444,6 +444,7 @@ cudaError_t launch_gram(const void* G, int dtype, int p, long long n, double* pa
   if (gram_tc_eligible(G, dtype, p, n)) return launch_gram_tc(G, p, n, partials, counter, K, status, st);
   if (gram_tm_eligible(G, dtype, p, n)) return launch_gram_tm(G, dtype, p, n, partials, counter, K, status, st);
   if (gram_tm32_eligible(G, dtype, p, n)) return launch_gram_tm32(G, p, n, partials, counter, K, status, st);
+  if (gram_tm64_eligible(G, dtype, p, n)) return launch_gram_tm64(G, p, n, partials, counter, K, status, st);
   const gram::Shape sh = gram::pick_shape(p);
   const int S = dtype == 0 ? 4 : 2;
   gram::Params prm{};

@@ -20,7 +20,9 @@
 // p <= 16: every warp takes whole tiles (tile u of a block goes to warp u mod 12) and loads them
 // itself; every thread keeps the upper triangle for its columns, as in fa_gram.cu; products in
 // fp32, runs of at most 64 columns, warp butterfly into fp64.  Block totals and the last-block reduction are
-// the ones of fa_gram.cu (bit-reproducible, single launch).
+// the ones of fa_gram.cu (bit-reproducible, single launch).  fp32 with 16 < p <= 32 and one row class has a
+// kernel of its own below (teams of four warps), and 32 < p <= 64 is put together from three launches by
+// row blocks of 32 (launch_gram_tm64).
 #include <atomic>
 
 #include "fa_gram_tm.cuh"
@@ -31,7 +33,10 @@ namespace fa {
 namespace gramtm {
 
 struct Params {
-  int p;
+  int p;                       // rows of the matrix this launch reads
+  int row0;                    // their position among the `ptotal` rows of K (a launch on a block of rows)
+  int ptotal;                  // rows of K
+  int finish;                  // the last block forms K from all blocks' sums (the last launch of a pass)
   long long num_tiles;
   double* partials;            // [p(p+1)/2][gridDim.x]
   unsigned int* counter;
@@ -180,10 +185,10 @@ gram_tri_tm_kernel(const __grid_constant__ Maps maps, const Params prm, const La
       // a block that gave up has incomplete sums: NaN, so that K comes out non-finite and whoever
       // reads it (the IRLS kernel sets FA_ST_NONFINITE and writes zeros) sees the failure
       if (*reinterpret_cast<volatile int*>(aborted)) sum = __longlong_as_double(0x7ff8000000000000LL);
-      prm.partials[(size_t)gram::canon_index(i, j, prm.p) * gridDim.x + blockIdx.x] = sum;
+      prm.partials[(size_t)gram::canon_index(prm.row0 + i, prm.row0 + j, prm.ptotal) * gridDim.x + blockIdx.x] = sum;
     }
   }
-  gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
+  if (prm.finish) gram::finish_gram(prm.partials, prm.counter, prm.K, prm.ptotal, flag);
 }
 
 // ---- 16 < p <= 32, one row class (rows on 16-byte boundaries), fp32.
@@ -363,9 +368,143 @@ gram_quad_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
     double sum = totals[(size_t)part * kQuadAcc + e] + totals[(size_t)(4 + part) * kQuadAcc + e];
     if (*reinterpret_cast<volatile int*>(&aborted[0]) | *reinterpret_cast<volatile int*>(&aborted[1]))
       sum = __longlong_as_double(0x7ff8000000000000LL);     // incomplete sums must not pass for inner products
+    prm.partials[(size_t)gram::canon_index(prm.row0 + gi, prm.row0 + gj, prm.ptotal) * gridDim.x + blockIdx.x] = sum;
+  }
+  if (prm.finish) gram::finish_gram(prm.partials, prm.counter, prm.K, prm.ptotal, flag);
+}
+
+// ---- 32 < p <= 64, one row class, fp32: the rectangle between rows 0-31 and rows 32..p-1.
+// K is put together from three launches over the same column tiles: the triangle kernel above on
+// rows 0-31, the same on rows 32..p-1, and this kernel for the 32 x (p - 32) entries between the two
+// blocks of rows -- the matrix is read twice, which is what 255 registers per thread allow (2080 sums
+// per column do not fit one block's registers, and sums have to stay in registers from tile to tile).
+// One tile holds all p rows (64 KB); the rectangle is cut into eight parts of 8 x 16 sums, one per
+// warp (a-rows 8 (w mod 4) .., b-rows 32 + 16 (w / 4) ..), operands by 4-byte loads of columns 32
+// apart as above.  All eight warps work on the same tile; the first thread re-issues a stage's load
+// behind the block's barrier.  This launch comes last and its last block forms K.
+constexpr int kCrossWarps = 8;
+constexpr int kCrossDepth = 3;               // stages of 64 KB
+constexpr int kCrossAcc = 128;
+
+__global__ void __launch_bounds__(kCrossWarps * 32, 1)
+gram_cross_tm_kernel(const __grid_constant__ Maps maps, const Params prm) {
+  constexpr int kThreads = kCrossWarps * 32;
+  constexpr int kRowBytes = kTileCols * 4;
+  constexpr int kStageBytes = 64 * kRowBytes;
+  extern __shared__ __align__(1024) char smem[];
+  char* stages = smem;
+  double* totals = reinterpret_cast<double*>(smem + (size_t)kCrossDepth * kStageBytes);
+  uint64_t* full = reinterpret_cast<uint64_t*>(totals + kCrossWarps * kCrossAcc);
+  int* flag = reinterpret_cast<int*>(full + kCrossDepth);
+  int* aborted = flag + 1;                   // a warp gave up on a tile
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) *aborted = 0;
+
+  for (int i = tid * 16; i < kCrossDepth * kStageBytes; i += kThreads * 16)
+    *reinterpret_cast<uint4*>(stages + i) = make_uint4(0, 0, 0, 0);
+  if (tid == 0)
+    for (int s = 0; s < kCrossDepth; ++s) mbar_init(&full[s], 1);
+  fence_proxy_async();
+  __syncthreads();
+
+  const uint32_t tile_bytes = static_cast<uint32_t>(prm.p * kRowBytes);
+  const int ntiles = static_cast<int>(prm.num_tiles);
+  const int tstride = static_cast<int>(gridDim.x);
+  const int tfirst = static_cast<int>(blockIdx.x);
+  auto issue = [&](int t, int s) {       // first thread of the block only
+    if (t >= ntiles) return;
+    mbar_arrive_expect_tx(&full[s], tile_bytes);
+    tma_load_2d(stages + (size_t)s * kStageBytes, &maps.map[0], t * kTileCols, 0, &full[s]);
+  };
+  const bool issuer = tid == 0;
+  if (issuer)
+    for (int v = 0; v < kCrossDepth; ++v) issue(tfirst + v * tstride, v);
+  // the loads in flight when the block gives up at tile t (stage s0, phase ph0) must land before it can
+  // exit: these waits keep the long limit
+  auto drain = [&](int t, int s0, uint32_t ph0) {
+    if (!issuer) return;
+    for (int k = 0; k < kCrossDepth; ++k) {
+      if (t + k * tstride < ntiles) (void)mbar_wait(&full[s0], ph0);
+      if (++s0 == kCrossDepth) { s0 = 0; ph0 ^= 1u; }
+    }
+  };
+
+  float acc[kCrossAcc];
+  double dacc[kCrossAcc / 32];
+#pragma unroll
+  for (int k = 0; k < kCrossAcc; ++k) acc[k] = 0.f;
+#pragma unroll
+  for (int k = 0; k < kCrossAcc / 32; ++k) dacc[k] = 0.0;
+  const int abase = 8 * (warp & 3) * kRowBytes;
+  const int bbase = (32 + 16 * (warp >> 2)) * kRowBytes;
+  const bool active = 32 + 16 * (warp >> 2) < prm.p;       // up to 48 rows the second half of the warps has no entries
+  int since = 0;
+  int s = 0;
+  uint32_t phase = 0;
+  for (int t = tfirst; t < ntiles; t += tstride) {
+    // giving up is a decision of the whole block, taken behind the barrier that ends the tile (as in the
+    // kernel above, with the block in the place of a team)
+    if (!__any_sync(0xffffffffu, mbar_wait(&full[s], phase, prm.wait_cycles))) {
+      if (lane == 0) {
+        if (prm.status) atomicOr(prm.status, kStTimeout);
+        *reinterpret_cast<volatile int*>(aborted) = 1;
+      }
+      __syncthreads();
+      drain(t, s, phase);
+      break;
+    }
+    const char* sbase = stages + (size_t)s * kStageBytes;
+#pragma unroll 1
+    for (int cg = active ? lane : kTileCols; cg < kTileCols; cg += 64) {
+      const char* pa = sbase + abase + cg * 4;
+      const char* pb = sbase + bbase + cg * 4;
+      float a[8][2], b[16][2];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        a[i][0] = *reinterpret_cast<const float*>(pa + i * kRowBytes);
+        a[i][1] = *reinterpret_cast<const float*>(pa + i * kRowBytes + 128);
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        b[j][0] = *reinterpret_cast<const float*>(pb + j * kRowBytes);
+        b[j][1] = *reinterpret_cast<const float*>(pb + j * kRowBytes + 128);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          acc[i * 16 + j] = fmaf(a[i][0], b[j][0], acc[i * 16 + j]);
+          acc[i * 16 + j] = fmaf(a[i][1], b[j][1], acc[i * 16 + j]);
+        }
+    }
+    __syncthreads();                     // all eight parts are done with the stage
+    if (*reinterpret_cast<volatile int*>(aborted)) {      // another warp gave up on this tile
+      drain(t, s, phase);
+      break;
+    }
+    if (issuer) {
+      fence_proxy_async();
+      issue(t + kCrossDepth * tstride, s);
+    }
+    if (++s == kCrossDepth) { s = 0; phase ^= 1u; }
+    since += 8;
+    if (since + 8 > kQuadFlushCols) { flush<kCrossAcc>(acc, dacc, lane); since = 0; }
+  }
+  flush<kCrossAcc>(acc, dacc, lane);
+#pragma unroll
+  for (int k = 0; k < kCrossAcc / 32; ++k) totals[warp * kCrossAcc + lane * (kCrossAcc / 32) + k] = dacc[k];
+  __syncthreads();
+
+  for (int idx = tid; idx < kCrossWarps * kCrossAcc; idx += kThreads) {
+    const int part = idx / kCrossAcc, e = idx - part * kCrossAcc;
+    const int gi = 8 * (part & 3) + e / 16, gj = 32 + 16 * (part >> 2) + e % 16;
+    if (gj >= prm.p) continue;
+    double sum = totals[idx];
+    if (*reinterpret_cast<volatile int*>(aborted))
+      sum = __longlong_as_double(0x7ff8000000000000LL);     // incomplete sums must not pass for inner products
     prm.partials[(size_t)gram::canon_index(gi, gj, prm.p) * gridDim.x + blockIdx.x] = sum;
   }
-  gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
+  if (prm.finish) gram::finish_gram(prm.partials, prm.counter, prm.K, prm.p, flag);
 }
 
 namespace {
@@ -459,6 +598,10 @@ bool gram_tm32_eligible(const void* G, int dtype, int p, long long n) {
   return dtype == 0 && p > 16 && p <= 32 && gramtm::available(G, dtype, n) && (n % 4) == 0;
 }
 
+bool gram_tm64_eligible(const void* G, int dtype, int p, long long n) {
+  return dtype == 0 && p > 32 && p <= 64 && gramtm::available(G, dtype, n) && (n % 4) == 0;
+}
+
 namespace {
 // Limit of the kernels' waits for a tile, in cycles.  Always kWaitCycles in normal use.
 std::atomic<long long> g_tile_wait_cycles{kWaitCycles};
@@ -483,6 +626,9 @@ cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials
   if (!gramtm::build(G, 0, p, n, maps, lay) || lay.q != 1) return cudaErrorInvalidValue;
   gramtm::Params prm{};
   prm.p = p;
+  prm.row0 = 0;
+  prm.ptotal = p;
+  prm.finish = 1;
   prm.num_tiles = (n + gramtm::kTileCols - 1) / gramtm::kTileCols;
   prm.partials = partials;
   prm.counter = counter;
@@ -502,24 +648,82 @@ cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials
   return cudaGetLastError();
 }
 
-cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
-                           double* K, int* status, cudaStream_t st) {
-  gramtm::Maps maps;
+namespace {
+// The p <= 16 kernel on the p rows at G; prm carries everything but p, the tile count and the wait limit.
+cudaError_t launch_tri_rows(const void* G, int dtype, int p, long long n, gramtm::Params prm, cudaStream_t st);
+}  // namespace
+
+cudaError_t launch_gram_tm64(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
+                             int* status, cudaStream_t st) {
+  const float* g = static_cast<const float*>(G);
+  const int rows2 = p - 32;
+  gramtm::Maps maps1, maps2, maps3;
   gramtm::Layout lay;
-  if (!gramtm::build(G, dtype, p, n, maps, lay)) return cudaErrorInvalidValue;
-  const int S = dtype == 0 ? 4 : 2;
+  if (!gramtm::build(g, 0, 32, n, maps1, lay) || lay.q != 1) return cudaErrorInvalidValue;
+  if (!gramtm::build(g + (size_t)32 * (size_t)n, 0, rows2, n, maps2, lay) || lay.q != 1) return cudaErrorInvalidValue;
+  if (!gramtm::build(g, 0, p, n, maps3, lay) || lay.q != 1) return cudaErrorInvalidValue;
   gramtm::Params prm{};
-  prm.p = p;
-  prm.num_tiles = (n + lay.step - 1) / lay.step;
+  prm.ptotal = p;
+  prm.num_tiles = (n + gramtm::kTileCols - 1) / gramtm::kTileCols;
   prm.partials = partials;
   prm.counter = counter;
   prm.K = K;
   prm.status = status;
   prm.wait_cycles = g_tile_wait_cycles.load();
   const int sms = sm_count();
-  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
+  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);     // the same for all three: one slot per block
+  const size_t smem_quad = (size_t)2 * gramtm::kQuadDepth * 32 * gramtm::kTileCols * 4 +
+                           (size_t)gramtm::kQuadWarps * gramtm::kQuadAcc * sizeof(double) +
+                           2 * gramtm::kQuadDepth * sizeof(uint64_t) + 64;
+  const size_t smem_cross = (size_t)gramtm::kCrossDepth * 64 * gramtm::kTileCols * 4 +
+                            (size_t)gramtm::kCrossWarps * gramtm::kCrossAcc * sizeof(double) +
+                            gramtm::kCrossDepth * sizeof(uint64_t) + 64;
+  cudaError_t e = cudaFuncSetAttribute(gramtm::gram_quad_tm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_quad);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(gramtm::gram_cross_tm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_cross);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
+  if (e != cudaSuccess) return e;
+  prm.p = 32; prm.row0 = 0; prm.finish = 0;
+  gramtm::gram_quad_tm_kernel<<<grid, gramtm::kQuadWarps * 32, smem_quad, st>>>(maps1, prm);
+  prm.p = rows2; prm.row0 = 32;
+  if (rows2 <= 16) {                    // a block of at most 16 rows goes through the faster kernel for such blocks
+    e = launch_tri_rows(g + (size_t)32 * (size_t)n, 0, rows2, n, prm, st);
+    if (e != cudaSuccess) return e;
+  } else {
+    gramtm::gram_quad_tm_kernel<<<grid, gramtm::kQuadWarps * 32, smem_quad, st>>>(maps2, prm);
+  }
+  prm.p = p; prm.row0 = 0; prm.finish = 1;
+  gramtm::gram_cross_tm_kernel<<<grid, gramtm::kCrossWarps * 32, smem_cross, st>>>(maps3, prm);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double* partials, unsigned int* counter,
+                           double* K, int* status, cudaStream_t st) {
+  gramtm::Params prm{};
+  prm.row0 = 0;
+  prm.ptotal = p;
+  prm.finish = 1;
+  prm.partials = partials;
+  prm.counter = counter;
+  prm.K = K;
+  prm.status = status;
   cudaError_t e = cudaMemsetAsync(counter, 0, sizeof(unsigned int), st);
   if (e != cudaSuccess) return e;
+  return launch_tri_rows(G, dtype, p, n, prm, st);
+}
+
+namespace {
+cudaError_t launch_tri_rows(const void* G, int dtype, int p, long long n, gramtm::Params prm, cudaStream_t st) {
+  gramtm::Maps maps;
+  gramtm::Layout lay;
+  if (!gramtm::build(G, dtype, p, n, maps, lay)) return cudaErrorInvalidValue;
+  const int S = dtype == 0 ? 4 : 2;
+  prm.p = p;
+  prm.num_tiles = (n + lay.step - 1) / lay.step;
+  prm.wait_cycles = g_tile_wait_cycles.load();
+  const int sms = sm_count();
+  const int grid = (int)(prm.num_tiles < sms ? prm.num_tiles : sms);
   const int pb = p <= 4 ? 4 : p <= 8 ? 8 : p <= 12 ? 12 : p <= 15 ? 15 : 16;
   const int naccp = (pb * (pb + 1) / 2 + 31) / 32 * 32;
   // two elements per shared load when every class's shift is even
@@ -535,5 +739,6 @@ cudaError_t launch_gram_tm(const void* G, int dtype, int p, long long n, double*
   if (dtype == 0) return gramtm::dispatch_tri<float>(pb, vec, maps, prm, lay, grid, smem, st);
   return gramtm::dispatch_tri<__nv_bfloat16>(pb, vec, maps, prm, lay, grid, smem, st);
 }
+}  // namespace
 
 }  // namespace fa

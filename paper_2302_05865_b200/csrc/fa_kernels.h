@@ -29,6 +29,11 @@ bool gram_tm32_eligible(const void* G, int dtype, int p, long long n);
 cudaError_t launch_gram_tm32(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
                              int* status, cudaStream_t st);
 
+// The same for fp32 with 32 < p <= 64: three launches (two triangles of 32 rows and the rectangle between them).
+bool gram_tm64_eligible(const void* G, int dtype, int p, long long n);
+cudaError_t launch_gram_tm64(const void* G, int p, long long n, double* partials, unsigned int* counter, double* K,
+                             int* status, cudaStream_t st);
+
 // Persistent single-block IRLS on K (p x p).
 struct IrlsArgs {
   const double* K;

@@ -19,7 +19,7 @@ from oracle import fa_oracle as fo
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("p,n,m", [(15, 300_002, 8), (31, 200_000, 12)])
+@pytest.mark.parametrize("p,n,m", [(15, 300_002, 8), (31, 200_000, 12), (40, 100_000, 12)])
 def test_a_wait_that_runs_out_is_reported_and_the_next_call_works(p, n, m):
     import paper_2302_05865_b200 as fa
     lib = ctypes.CDLL(fa.LIB_PATH)

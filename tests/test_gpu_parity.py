@@ -55,6 +55,9 @@ LADDER = [
     # of columns half a tile apart; the tile step is 256 or 252 columns)
     (13, 20_001, "noisy_mean", False, 0), (14, 30_002, "gauss", False, 0), (16, 50_003, "dup_zero", False, 0),
     (16, 40_002, "noisy_mean", False, 2), (13, 8_192, "gauss", False, 4),
+    # fp32, 32 < p <= 64, rows on 16-byte boundaries: two triangle launches and the rectangle between the row blocks
+    (48, 100_000, "noisy_mean", False, 0), (63, 40_004, "dup_zero", False, 0), (64, 8_192, "gauss", False, 0),
+    (40, 4_096, "gauss", False, 4), (34, 300_000, "noisy_mean", False, 0), (57, 1_000_000, "gauss", False, 8),
     # bf16, p > 16, 16-byte aligned rows: the tensor-core kernel
     (17, 64, "gauss", True, 0), (33, 264, "noisy_mean", True, 0), (63, 4_096, "dup_zero", True, 0),
     (64, 65_536, "gauss", True, 0), (31, 1_000_000, "dup_zero", True, 8), (48, 300_008, "noisy_mean", True, 0),
@@ -307,6 +310,7 @@ AGG_LADDER = [
     (15, 100_003, "noisy_mean", True, 8, 0.01, 8, 0), (31, 40_002, "noisy_mean", True, 12, 0.02, 8, 2),
     (63, 66_000, "dup_zero", True, 16, 0.01, 8, 0), (33, 264, "noisy_mean", True, 10, 0.02, 6, 0),
     (64, 65_536, "noisy_mean", True, 20, 0.01, 6, 0), (31, 1_000_000, "dup_zero", True, 12, 0.01, 8, 8),
+    (48, 100_000, "noisy_mean", False, 16, 0.01, 6, 0), (63, 40_004, "dup_zero", False, 16, 0.02, 6, 4),
 ]
 
 
