@@ -350,18 +350,18 @@ def main():
         comb_gbs = comb_bytes / (t_comb * 1e-3) / 1e9
         step_gbs = w_full.algorithmic_bytes / (ms_per_step * 1e-3) / 1e9
         # DRAM bytes of one Gram launch, from ncu captures of the kernels as they stand, on cases small enough to
-        # capture: fp32 p = 15 at n = 4,000,002 (rows in two alignment classes, as in the full workload): 240.12 MB
-        # read for 240.00 MB of gradients, 9.9 MB written; fp32 p = 31 at n = 2,000,000: 248.11 MB read for
-        # 248.00 MB, 3.7 MB written.  The reads grow with n; the writes are per block and do not.
+        # capture: fp32 p = 15 at n = 4,000,002 (rows in two alignment classes, as in the full workload): 240.11 MB
+        # read for 240.00 MB of gradients, 8.8 MB written; fp32 p = 31 at n = 2,000,000: 248.10 MB read for
+        # 248.00 MB, 4.0 MB written.  The reads grow with n; the writes are per block and do not.
         traffic, traffic_source = None, None
         if w.p == 15 and w.dtype == "f32" and w.n >= 4096:
-            traffic = int(240.117e6 * (w.n / 4_000_002) + 9.9e6)
+            traffic = int(240.110e6 * (w.n / 4_000_002) + 8.8e6)
             traffic_source = ("ncu capture of gramtm::gram_tri_tm_kernel<float,2,15> at n = 4,000,002 "
-                              "(dram__bytes_read 240.12 MB, dram__bytes_write 9.9 MB); reads scaled by n, writes not")
+                              "(dram__bytes_read 240.11 MB, dram__bytes_write 8.8 MB); reads scaled by n, writes not")
         elif w.p == 31 and w.dtype == "f32" and w.n >= 4096:
-            traffic = int(248.11e6 * (w.n / 2_000_000) + 3.7e6)
+            traffic = int(248.10e6 * (w.n / 2_000_000) + 4.0e6)
             traffic_source = ("ncu capture of gram_quad_tm_kernel at n = 2,000,000 "
-                              "(dram__bytes_read 248.11 MB, dram__bytes_write 3.7 MB); reads scaled by n, writes not")
+                              "(dram__bytes_read 248.10 MB, dram__bytes_write 4.0 MB); reads scaled by n, writes not")
         roofline = {"kernel": "gram pass (K = G G^T)", "bound": "hbm", "achieved": gram_gbs, "peak": peak,
                     "unit": "GB/s", "frac": gram_gbs / peak, "frac_of_nominal_8TBs": gram_gbs / 8000.0,
                     "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_src,
