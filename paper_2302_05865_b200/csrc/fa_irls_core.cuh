@@ -26,9 +26,14 @@
 #ifndef FA_IRLS_HOST
 #define FA_FN __device__ __forceinline__
 #define FA_HD __host__ __device__ inline
+// A function that is called from several places and is large, or that only rare arguments reach: one copy,
+// out of line.  The kernels' code does not fit the instruction cache (stalls for instruction fetch were
+// a fifth of all stall cycles at 15 gradients), so every copy that is not needed is paid for in time.
+#define FA_FN_SHARED __device__ __noinline__
 #else
 #define FA_FN static inline
 #define FA_HD static inline
+#define FA_FN_SHARED static
 #endif
 
 #ifndef FA_IRLS_HOST
@@ -234,6 +239,7 @@ FA_FN double dot(const double* a, const double* b, int n) {
       for (int u = 0; u < CH; u += 2) { acc0 = fma(x[u], y[u], acc0); acc1 = fma(x[u + 1], y[u + 1], acc1); }
     }
   } else {
+#pragma unroll 1
     for (int k0 = 0; k0 < n; k0 += CH, a += CH * SA, b += CH * SB) {
       double x[CH], y[CH];
 #pragma unroll
@@ -253,6 +259,7 @@ template <int SA, int SB, int NMAX>
 FA_FN double dot_weighted(const double* w, const double* a, const double* b, int n) {
   constexpr int CH = 8;
   double acc0 = 0.0, acc1 = 0.0;
+#pragma unroll 1
   for (int k0 = 0; k0 < n; k0 += CH, w += CH, a += CH * SA, b += CH * SB) {
     double x[CH], y[CH];
 #pragma unroll
@@ -272,6 +279,7 @@ template <int ST>
 FA_FN void diff_sq(const double* a, const double* b, int k0, int n, double& all, double& tail) {
   constexpr int CH = 8;
   double s0 = 0.0, s1 = 0.0, t0 = 0.0, t1 = 0.0;
+#pragma unroll 1
   for (int kb = 0; kb < n; kb += CH, a += CH * ST, b += CH * ST) {
     double v[CH];
 #pragma unroll
@@ -317,6 +325,7 @@ FA_FN void matmul(const Ctx& c, int M, int N, int K, const FastDiv& dtn, const d
   const int warp = ((c.tid >> 5) - first_warp) & (nwarp - 1);
   const int tn = (N + 7) >> 3, tiles = ((M + 7) >> 3) * tn;
   const int fr = lane >> 2, fk = lane & 3;          // fragment coordinates: A (row fr, k fk), B (k fk, column fr)
+#pragma unroll 1
   for (int t = warp; t < tiles; t += nwarp) {
     const int ti = fast_div(t, dtn);
     const int i0 = ti * 8, j0 = (t - ti * tn) * 8;
@@ -326,6 +335,7 @@ FA_FN void matmul(const Ctx& c, int M, int N, int K, const FastDiv& dtn, const d
     const double* ap = A + ia * SAI + fk * SAK;
     const double* bp = B + fk * SBK + jb * SBJ;
     double d0 = 0.0, d1 = 0.0, e0 = 0.0, e1 = 0.0;  // two chains of dependent instructions, added at the end
+#pragma unroll 1
     for (int k0 = 0; k0 < K; k0 += 16, ap += 16 * SAK, bp += 16 * SBK) {
       double a[4], b[4];
 #pragma unroll
@@ -351,6 +361,7 @@ FA_FN void matmul(const Ctx& c, int M, int N, int K, const FastDiv& dtn, const d
   }
 #else
   (void)first_warp; (void)dtn;
+#pragma unroll 1
   for (int idx = c.tid; idx < M * N; idx += c.nt) {
     const int i = idx / N, j = idx - i * N;
     const int ia = imap ? imap[i] : i, jb = jmap ? jmap[j] : j;
@@ -590,6 +601,7 @@ FA_FN int jacobi_small(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
       }
 #endif
       // further items (fewer threads than items): offsets on the fly
+#pragma unroll 1
       for (int idx = c.tid + c.nt; idx < total2; idx += c.nt) {
         if (idx < nb2) {
           const int k = idx / np, l = idx - k * np;
@@ -734,6 +746,7 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
       if (!kOnce && lane < np) { s.rc[lane] = (double)cq; s.rs[lane] = (double)sq; }     // same values from every warp: for the loops below
       // items beyond the per-thread lists (a smaller block than expected): offsets on the fly
       if (!kOnce && (kMT * c.nt < np * np || kMJ * c.nt < jrows * np)) c.sync();
+#pragma unroll 1
       for (int idx = c.tid + kMT * c.nt; idx < np * np; idx += c.nt) {
         const int k = idx / np, l = idx - k * np;
         const int a = k, b = np + k, cc = l, d = np + l;
@@ -746,6 +759,7 @@ FA_FN int jacobi_large(const Ctx& c, const Smem& s, R** Tio, R** Taltio, R** Jio
         Tn[pa * ld + pc] = cl * yac - sl * yad; Tn[pa * ld + pd] = sl * yac + cl * yad;
         Tn[pb * ld + pc] = cl * ybc - sl * ybd; Tn[pb * ld + pd] = sl * ybc + cl * ybd;
       }
+#pragma unroll 1
       for (int idx = c.tid + kMJ * c.nt; idx < jrows * np; idx += c.nt) {
         const int x = idx / np, l = idx - x * np;
         const int cc = l, d = np + l;
@@ -829,6 +843,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
   int steps = 0;
   if (!from_x) {
     // ---- first step from X = I
+#pragma unroll 1
     for (int idx = c.tid; idx < r * r; idx += c.nt) {
       const int i = fast_div(idx, s.div_r), j = idx - i * r;
       double e = 0.0;
@@ -843,6 +858,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
     }
     emax = block_max(c, s, part);                      // its barrier also publishes X
     if (!(emax <= kRefineTheta)) return 0;
+#pragma unroll 1
     for (int k = c.tid; k < r; k += c.nt) s.lam[k] = T[k * ld + k];
     steps = 1;
   }
@@ -873,6 +889,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
     // ---- the correction.  lam_i = S_ii / (1 - Rm_ii) with the quotient expanded to second order:
     // Rm_ii is of the order of the last correction squared.
     part = 0.0;
+#pragma unroll 1
     for (int idx = c.tid; idx < r * r; idx += c.nt) {
       const int i = fast_div(idx, s.div_r), j = idx - i * r;
       const double rii = s.rdiag[i];
@@ -907,6 +924,7 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
     ++steps;
   }
   c.sync();
+#pragma unroll 1
   for (int k = c.tid; k < r; k += c.nt) s.T[k * ld + k] = s.lam[k];
   s.J = X; s.M = SR;
   s.count_refinements += steps;
@@ -931,9 +949,11 @@ FA_FN void sweeps_fp32(const Ctx& c, Smem& s, int r) {
   float* Jf = reinterpret_cast<float*>(s.M);
   float* Ja = Jf + (LD - kLdPad) * LD;
   double part = 0.0;
+#pragma unroll 1
   for (int k = c.tid; k < r; k += c.nt) part = fmax(part, fmin(fabs(s.T[k * ld + k]), 1.7e308));
   const double dmax = block_max(c, s, part);
   const double scale = dmax > 0.0 ? 1.0 / dmax : 1.0;
+#pragma unroll 1
   for (int idx = c.tid; idx < ppr * ld; idx += c.nt) {
     const int a = idx / ld, b = idx - a * ld;          // ld is a compile-time constant
     Tf[idx] = (a < r && b < r) ? (float)(s.T[idx] * scale) : 0.0f;
@@ -945,6 +965,7 @@ FA_FN void sweeps_fp32(const Ctx& c, Smem& s, int r) {
     s.count_sweeps_f32 += jacobi<LD, float>(c, s, &Tf, &Ta, &Jf, &Ja, r, r, 1, &big);
     if (!big) break;
     part = 0.0;
+#pragma unroll 1
     for (int idx = c.tid; idx < r * r; idx += c.nt) {
       const int i = fast_div(idx, s.div_r), j = idx - i * r;
       if (i != j) {
@@ -957,6 +978,7 @@ FA_FN void sweeps_fp32(const Ctx& c, Smem& s, int r) {
     }
     if (block_max(c, s, part) <= 0.5 * RefineLimits<LD>::theta) break;
   }
+#pragma unroll 1
   for (int idx = c.tid; idx < r * r; idx += c.nt) {
     const int i = fast_div(idx, s.div_r), j = idx - i * r;
     s.J[i * ld + j] = (double)Jf[i * ld + j];
@@ -976,6 +998,7 @@ FA_FN int sort_eigs(const Ctx& c, const Smem& s, const double* T, int dim, int l
 #ifdef FA_IRLS_HOST
   int keep = 0;
 #endif
+#pragma unroll 1
   for (int k = c.tid; k < dim; k += c.nt) {
     const double e = T[k * ld + k];
     double top = e;
@@ -1002,10 +1025,13 @@ FA_FN int sort_eigs(const Ctx& c, const Smem& s, const double* T, int dim, int l
 // One term of the objective with value u (the quantity under the root in Eq. (5)): its
 // contribution u^(1/a) and the factor max(u^(1 - 1/a), eps) of its reweighting (Eq. (4) with
 // constant a; a = 2 gives the square roots of Eq. (5) and takes the sqrt fast path).
+FA_FN_SHARED void term_of_general(double u, double a, double& contrib, double& denom) {
+  if (u <= 0.0) { contrib = 0.0; denom = kEps; }
+  else { contrib = pow(u, 1.0 / a); denom = fmax(pow(u, 1.0 - 1.0 / a), kEps); }
+}
 FA_FN void term_of(double u, double a, double& contrib, double& denom) {
   if (a == 2.0) { contrib = sqrt(u); denom = fmax(contrib, kEps); }
-  else if (u <= 0.0) { contrib = 0.0; denom = kEps; }
-  else { contrib = pow(u, 1.0 / a); denom = fmax(pow(u, 1.0 - 1.0 / a), kEps); }
+  else term_of_general(u, a, contrib, denom);
 }
 
 // From residual coordinates Res (rows k0..r-1 are the part of f_i outside the subspace) and the
@@ -1021,6 +1047,7 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
                                    bool want_objective = true) {
   constexpr int ld = LD;
   double part = 0.0;
+#pragma unroll 1
   for (int i = c.tid; i < p; i += c.nt) {
     double ui = 0.0, wi = 0.0;
     if (s.dinv[i] != 0.0) {
@@ -1070,6 +1097,7 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
   if (coef > 0.0) {
     // off-diagonal entries M_ij = M_ji = -2 w_ij (ordered pairs: each unordered pair counted twice, and
     // twice in the objective); one item per unordered pair i < j
+#pragma unroll 1
     for (int idx = c.tid; idx < p * (p - 1) / 2; idx += c.nt) {
       const int i = s.pairs[idx] >> 8, j = s.pairs[idx] & 255;
       double d2, res2;
@@ -1096,6 +1124,7 @@ FA_FN double weights_and_objective(const Ctx& c, Smem& s, const double* Res, int
       s.M[j * ld + i] = -2.0 * wij;
     }
     c.sync();
+#pragma unroll 1
     for (int i = c.tid; i < p; i += c.nt) {
       double acc = 0.0;
       for (int j = 0; j < p; ++j) acc -= (j != i) ? s.M[i * ld + j] : 0.0;
@@ -1124,6 +1153,7 @@ FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* 
   double part = 0.0;
   double gmax = 0.0;
   for (int i = 0; i < nw; ++i) gmax = fmax(gmax, s.gtr[i]);
+#pragma unroll 1
   for (int i = c.tid; i < nw; i += c.nt) {
     double ui = 0.0, wi = 0.0;
     if (s.gtr[i] > kZeroNormRel * gmax) {
@@ -1144,6 +1174,7 @@ FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* 
     s.gw[i] = wi;
   }
   if (coef > 0.0) {
+#pragma unroll 1
     for (int idx = c.tid; idx < r * nw; idx += c.nt) {
       const int k = idx / nw, i = idx - k * nw;
       const int r0 = s.first[i], r1 = (i + 1 < nw) ? s.first[i + 1] : p;
@@ -1154,9 +1185,11 @@ FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* 
     }
   }
   c.sync();
+#pragma unroll 1
   for (int row = c.tid; row < p; row += c.nt) { s.w[row] = s.gw[s.grp[row]]; s.u[row] = s.gu[s.grp[row]]; }
   if (coef > 0.0) {
     // rows of different workers i != j: M = -2 w_ij / (k_i k_j)  (ordered pairs: each pair twice)
+#pragma unroll 1
     for (int idx = c.tid; idx < p * p; idx += c.nt) {
       const int ra = idx / p, rb = idx - ra * p;
       const int i = s.grp[ra], j = s.grp[rb];
@@ -1181,6 +1214,7 @@ FA_FN double weights_and_objective_grouped(const Ctx& c, Smem& s, const double* 
     }
     c.sync();
     // rows of one worker: what makes the pair part's row sums vanish, plus the data weight
+#pragma unroll 1
     for (int idx = c.tid; idx < p * p; idx += c.nt) {
       const int ra = idx / p, rb = idx - ra * p;
       const int i = s.grp[ra];
@@ -1204,10 +1238,15 @@ struct Outputs {
 };
 
 FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int iters, int nweights) {
+#pragma unroll 1
   for (int i = c.tid; i < p * m; i += c.nt) if (o.A) o.A[i] = 0.0;
+#pragma unroll 1
   for (int i = c.tid; i < p; i += c.nt) if (o.c) o.c[i] = 0.f;
+#pragma unroll 1
   for (int i = c.tid; i < nweights; i += c.nt) if (o.w) o.w[i] = 0.0;
+#pragma unroll 1
   for (int i = c.tid; i < iters; i += c.nt) if (o.obj) o.obj[i] = 0.0;
+#pragma unroll 1
   for (int i = c.tid; i < p * p; i += c.nt) if (o.S) o.S[i] = 0.0;
   if (o.rounds && c.tid == 0) *o.rounds = 0;
 }
@@ -1231,8 +1270,10 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   if (c.tid == 0) { s.flags[1] = 0; }
   s.div_p = make_div(p);
   c.sync();
+#pragma unroll 1
   for (int idx = c.tid; idx < pp * ld; idx += c.nt) { s.T[idx] = 0.0; s.J[idx] = 0.0; s.Aacc[idx] = 0.0; s.P[idx] = 0.0; s.M[idx] = 0.0; s.tmp[idx] = 0.0; }
   c.sync();
+#pragma unroll 1
   for (int idx = c.tid; idx < p * p; idx += c.nt) {
     const int i = fast_div(idx, s.div_p), j = idx - i * p;
     double v = K[idx];
@@ -1250,12 +1291,14 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     write_zero_outputs(c, o, p, m, iters, nw > 0 ? nw : p);
     return ST_RANK0;
   }
+#pragma unroll 1
   for (int idx = c.tid; idx < p * (p - 1) / 2; idx += c.nt) {
     int i, jm;
     tri_pair(idx, i, jm);                         // i <= jm over p - 1 columns: the pair (i, jm + 1)
     s.pairs[idx] = (unsigned short)((i << 8) | (jm + 1));
   }
   // kd = ||g_i||^2, dinv = 1 / ||g_i|| (0 for a zero gradient), fn (for now) = ||g_i||
+#pragma unroll 1
   for (int i = c.tid; i < p; i += c.nt) {
     const double kii = s.T[i * ld + i];
     const bool zero = kii <= kZeroNormRel * kmax;
@@ -1265,6 +1308,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   c.sync();
 
   // ---- Kt = D^-1 K D^-1 (symmetrised, unit diagonal) -> tmp
+#pragma unroll 1
   for (int idx = c.tid; idx < p * (p + 1) / 2; idx += c.nt) {
     int i, j;
     tri_pair(idx, i, j);
@@ -1274,6 +1318,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   }
   // remaining diagonal of the factorisation -> u (and, on alternate steps, w: see below); ord[j] = 0
   // while column j has not been a pivot, else 1 + the step at which it was
+#pragma unroll 1
   for (int i = c.tid; i < p; i += c.nt) { s.u[i] = (s.dinv[i] != 0.0) ? 1.0 : 0.0; s.ord[i] = 0; }
   c.sync();
 
@@ -1317,6 +1362,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     const double dpiv = ucur[piv];
     if (!(dpiv > kRankRel)) break;                // (the upper-word test lets a value just below the cut through)
     const double rinv = FA_RSQRT(dpiv), rkk = dpiv * rinv;   // dpiv in (1e-12, 1]: a normal number
+#pragma unroll 1
     for (int j = c.tid; j < p; j += c.nt) {
       const int mark = s.ord[j];
       const bool done = mark != 0 && mark <= k;   // a pivot of an earlier step
@@ -1340,11 +1386,13 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   // per thread -> J buffer.  Q = G D^-1 X with X[piv_a][:] = U[a][:] has orthonormal columns and
   // Q^T g_i = f_i, so Aacc starts as D^-1 X (p x r).  First the pivot columns are gathered (-> M),
   // so that the sums below run over consecutive elements; 1 / R11_aa is the rinv of step a.
+#pragma unroll 1
   for (int idx = c.tid; idx < r * r; idx += c.nt) {
     const int a = fast_div(idx, s.div_r), l = idx - a * r;
     s.M[a * ld + l] = s.P[a * ld + s.piv[l]];
   }
   c.sync();
+#pragma unroll 1
   for (int bcol = c.tid; bcol < r; bcol += c.nt) {
     for (int a = bcol; a >= 0; --a) {
       const double sum = dot<1, LD, LD - kLdPad>(s.M + a * ld + a + 1, s.J + (a + 1) * ld + bcol, bcol - a);
@@ -1352,6 +1400,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
   }
   c.sync();
+#pragma unroll 1
   for (int idx = c.tid; idx < r * r; idx += c.nt) {
     const int a = fast_div(idx, s.div_r), bcol = idx - a * r;
     if (bcol >= a) {
@@ -1360,12 +1409,14 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
   }
   // ---- P = F: scale column i of R back by ||g_i||; fn = ||f_i||^2
+#pragma unroll 1
   for (int i = c.tid; i < p; i += c.nt) {
     const double nrm = s.fn[i];
     double acc = 0.0;
     for (int k = 0; k < r; ++k) { const double v = s.P[k * ld + i] * nrm; s.P[k * ld + i] = v; acc = fma(v, v, acc); }
     s.fn[i] = acc;
   }
+#pragma unroll 1
   for (int idx = c.tid; idx < pp * ld; idx += c.nt) s.M[idx] = 0.0;     // M held the gathered columns
   c.sync();
   int sw = 0;
@@ -1384,6 +1435,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       }
     }
     c.sync();
+#pragma unroll 1
     for (int i = c.tid; i < nw; i += c.nt) {
       const int r0 = s.first[i], r1 = (i + 1 < nw) ? s.first[i + 1] : p;
       double acc = 0.0;
@@ -1398,6 +1450,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   // ---- weights of the first round
   if (start != 0) {
     // Z0 = F A0 (r x m) -> J buffer
+#pragma unroll 1
     for (int idx = c.tid; idx < r * m; idx += c.nt) {
       int k = idx / m, q = idx - k * m;
       double acc = 0.0;
@@ -1407,6 +1460,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     c.sync();
     if (start == 2) {
       // W = Z0^T Z0 -> T; Cholesky W = L L^T by one thread; Z = Z0 L^-T row by row
+#pragma unroll 1
       for (int idx = c.tid; idx < m * m; idx += c.nt) {
         int q = idx / m, l = idx - q * m;
         double acc = 0.0;
@@ -1435,6 +1489,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       c.sync();
       if (s.flags[1] == 0) start = 0;
       else {
+#pragma unroll 1
         for (int k = c.tid; k < r; k += c.nt) {
           for (int q = 0; q < m; ++q) {
             double v = s.J[k * ld + q];
@@ -1451,6 +1506,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     else (void)weights_and_objective<LD>(c, s, s.P, 0, r, p, coef, true, a, cb, ca);
   } else {
     // C = Z0^T F (m x p) -> T buffer; Res = F - Z0 C -> tmp
+#pragma unroll 1
     for (int idx = c.tid; idx < m * p; idx += c.nt) {
       int q = idx / p, i = idx - q * p;
       double acc = 0.0;
@@ -1458,6 +1514,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       s.T[q * ld + i] = acc;
     }
     c.sync();
+#pragma unroll 1
     for (int idx = c.tid; idx < r * p; idx += c.nt) {
       int k = idx / p, i = idx - k * p;
       double acc = s.P[k * ld + i];
@@ -1473,6 +1530,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
   double prev_obj = 0.0;
   for (int t = 0; t < iters; ++t) {
     sw = 0;
+#pragma unroll 1
     for (int i = c.tid; i < p; i += c.nt) s.wused[i] = s.w[i];
     if (grouped) for (int i = c.tid; i < nw; i += c.nt) s.gwused[i] = s.gw[i];
     // ---- T = P M P^T (current basis); only one triangle is taken from the product, so that T is
@@ -1483,6 +1541,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       matmul<LD, 1, LD, 1>(c, r, r, p, s.div_tr, s.P, s.tmp,
                            [&](int a, int b, double v) { if (a <= b) { s.T[a * ld + b] = v; s.T[b * ld + a] = v; } });
     } else {
+#pragma unroll 1
       for (int idx = c.tid; idx < r * p; idx += c.nt) {                                   // tmp = P diag(w)
         const int a = fast_div(idx, s.div_p), i = idx - a * p;
         s.tmp[a * ld + i] = s.w[i] * s.P[a * ld + i];
@@ -1508,9 +1567,11 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
         if (refine_eig<LD>(c, s, r, true)) break;
       }
       const int ppr = (r + 1) & ~1;                       // the sweeps work on an even number of indices
+#pragma unroll 1
       for (int idx = c.tid; idx < ppr * ld; idx += c.nt) s.J[idx] = 0.0;
       if (ppr > r) for (int b = c.tid; b < ppr; b += c.nt) { s.T[r * ld + b] = 0.0; s.T[b * ld + r] = 0.0; }
       c.sync();
+#pragma unroll 1
       for (int a = c.tid; a < ppr; a += c.nt) s.J[a * (ld + 1)] = 1.0;
       c.sync();
       int big = 0;
@@ -1553,6 +1614,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
 
   // ---- outputs
   if (o.A) {
+#pragma unroll 1
     for (int idx = c.tid; idx < p * m; idx += c.nt) {
       int i = idx / m, q = idx - i * m;
       o.A[idx] = (q < m_eff) ? s.Aacc[i * ld + q] : 0.0;
@@ -1563,6 +1625,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     else for (int i = c.tid; i < p; i += c.nt) o.w[i] = s.wused[i];
   }
   if (o.S) {   // Y Y^T G = G S with S = A (A^T K): (A^T K) e_j are the leading coordinates of f_j
+#pragma unroll 1
     for (int idx = c.tid; idx < p * p; idx += c.nt) {
       const int i = idx / p, j = idx - i * p;
       double acc = 0.0;
@@ -1571,6 +1634,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
     }
   }
   if (o.c) {
+#pragma unroll 1
     for (int k = c.tid; k < m_eff; k += c.nt) {        // s_k = sum_j P[k][j]  (Z^T F 1)
       double acc = 0.0;
       if (grouped) for (int j = 0; j < p; ++j) acc += s.P[k * ld + j] * s.ginv[s.grp[j]];   // sum of worker means
@@ -1578,6 +1642,7 @@ FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambd
       s.ev[k] = acc;
     }
     c.sync();
+#pragma unroll 1
     for (int i = c.tid; i < p; i += c.nt) {
       double acc = 0.0;
       for (int k = 0; k < m_eff; ++k) acc += s.Aacc[i * ld + k] * s.ev[k];
