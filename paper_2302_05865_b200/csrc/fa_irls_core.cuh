@@ -1258,10 +1258,15 @@ FA_FN void write_zero_outputs(const Ctx& c, const Outputs& o, int p, int m, int 
 // first, and a rank-deficient one falls back to the uniform round.  tol >= 0: stop after round
 // t >= 2 once the objective moved by <= tol (remaining entries of o.obj repeat the last value).  nw > 0: the p rows belong to nw workers, cnt[i] consecutive rows each (o.w then has nw
 // entries); nw = 0: one gradient per worker.  Returns the status bits (same value in every thread).
-template <int LD>
+// kPlain: the caller promises the paper's default terms (a = 2, Beta(1, 1/2), one gradient per worker).  The
+// arguments are then replaced by those constants, the compiler drops every other branch, and the code of
+// a round shrinks to what this case executes -- the kernels are bound by instruction fetch as much as by
+// anything else (their code does not fit the instruction cache).
+template <int LD, bool kPlain = false>
 FA_FN int run(const Ctx& c, Smem& s, const double* K, int p, int m, double lambda, double a, int iters,
               int start, const double* A0, double tol, const Outputs& o, int nw = 0,
               const unsigned char* cnt = nullptr, double cb = 1.0, double ca = 0.0) {
+  if (kPlain) { a = 2.0; nw = 0; cnt = nullptr; cb = 1.0; ca = 0.0; }
   constexpr int ld = LD;
   const int pp = (p + 1) & ~1;
   int status = 0;
