@@ -837,7 +837,6 @@ FA_FN int refine_eig(const Ctx& c, Smem& s, int r, bool from_x = false) {
   double* X = s.J;       // current eigenvector estimate
   double* E = s.tmp;     // T X, then the correction E
   double* SR = s.M;      // S on and above the diagonal, Rm below it; becomes the next X
-  const int ntri = r * (r + 1) / 2;
   constexpr double kRefineTheta = RefineLimits<LD>::theta, kRefineContract = RefineLimits<LD>::contract;
   double part = 0.0, emax = kRefineTheta / kRefineContract;   // from_x: the first full step must come out below kRefineTheta
   int steps = 0;
