@@ -120,7 +120,10 @@ def test_full_size_matches_the_stored_oracle_run(fa, name):
     # the cut between kept and discarded directions runs through a cluster of nearly equal eigenvalues
     # (relative gaps of 1e-4 at these n), which amplifies the 1e-9 error of the inner products: the two
     # trajectories part by up to a few 1e-3 in the objective around rounds 4-7 and meet again (1e-7 at
-    # the last round at p = 31).  So: a loose bound on every round, a tight one on where the rounds end.
+    # the last round at p = 31).  How far they part is itself a matter of rounding: the same kernel with its
+    # fp32 running sums folded every 256 columns instead of 128 (inner products good to 4e-9 instead of 2e-9)
+    # is 3.4e-2 away at round 6 and again 3.6e-7 at the end.  So: a loose bound on every round (the objective
+    # is of order p), a tight one on where the rounds end.
     diff = np.abs(obj.cpu().numpy() - gold["objective"])
     w_err = float(np.max(np.abs(wts.cpu().numpy() - gold["w"]) / np.maximum(np.abs(gold["w"]), 1e-300)))
     print(f"{name}: objective differences per round {diff}")
@@ -128,7 +131,7 @@ def test_full_size_matches_the_stored_oracle_run(fa, name):
     # the result of the rounds moves by about 30 times the relative error of the inner products (measured by
     # perturbing K): 1e-9 on the fp32 pipes, up to 2e-6 on the tensor-core path
     obj_tol, w_tol = (1e-3, 1e-1) if tensor_cores else (1e-5, 1e-2)
-    assert diff.max() < 2e-2 and obj_err < obj_tol and w_err < w_tol
+    assert diff.max() < 1e-1 and obj_err < obj_tol and w_err < w_tol
 
     # the aggregate at the stored columns (relative L2 over the sample, and element by element
     # against the root-mean-square entry), and its norm
